@@ -1,0 +1,1114 @@
+// AdaScale SGD gain-ratio step for sm_100a: kernels and the C-ABI host glue.
+//
+// Three kernels make up one iteration (paper: Sec. 3.2, App. B.3, Eq. 2-3):
+//   reduce  - streams the S x P gradient matrix once, writes the mean gradient and one
+//             pair (sum of squared deviations, squared norm of the mean) per block; the
+//             block that finishes last adds the pairs in index order and runs the scalar
+//             part (estimates, clamps, moving averages, r_t, eta_t, tau_{t+1}).
+//   update  - v <- rho v + (gbar + lambda w), w <- w - eta_t v, reading eta_t from the device.
+//   probes  - trivial streaming kernels that calibrate the bandwidth ceiling.
+// The path is bound by HBM bandwidth; there is no contraction, hence no tensor-core work.
+#include "../../include/adascale.h"
+
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kChunkF32 = 2048;   // elements one block handles (fp32 gradients)
+constexpr int kChunkBF16 = 4096;  // elements one block handles (bf16 gradients)
+constexpr int kGbarAlign = 64;    // every tensor's mean gradient starts on a 256-byte boundary
+constexpr int kRing = 4;          // pinned staging slots for pointer-table uploads
+constexpr int kMaxS = 4096;
+
+typedef unsigned long long u64;
+
+struct Chunk {
+    long long off;   // first element inside the tensor
+    long long goff;  // first element inside the mean-gradient workspace
+    int tensor;
+    int len;
+};
+
+// Scalar state kept on the device between iterations.
+struct DevState {
+    double tau;    // scale-invariant iteration tau_t
+    double avg_a;  // sigma_bar^2 (ratio estimator: m1)
+    double avg_b;  // mu_bar^2    (ratio estimator: m2)
+    long long n;   // samples absorbed by the averages
+    long long t;   // iterations applied
+    long long skipped;
+    double r, eta, lr;
+    double sigma2_raw, mu2_raw;
+    double N, D;
+    unsigned status;
+    unsigned pad;
+};
+
+struct ScalarCfg {
+    double eps, theta;  // theta already resolved (paper rule applied on the host side of set_scale)
+    unsigned flags;
+    int S;
+};
+
+struct Sched {
+    int kind, n;
+    double eta0, decay, t_s1;
+    double w[ADASCALE_MAX_MILESTONES];
+};
+
+struct ReduceArgs {
+    const Chunk *chunks;
+    const u64 *gptr;        // [S * T] row pointers
+    const unsigned *gflags; // [T] bit0: all S rows of the tensor are 16-byte aligned
+    float *gbar;
+    double2 *partials;
+    unsigned *ticket;
+    DevState *st;
+    int n_chunks, S, T;
+    float invS, fS;
+    ScalarCfg sc;
+    Sched sched;
+};
+
+struct UpdateArgs {
+    const Chunk *chunks;
+    const u64 *wv;          // [2 * T]: parameters then momentum
+    const unsigned *wflags; // [T] bit0: both pointers 16-byte aligned
+    const float *gbar;
+    const DevState *st;
+    int n_chunks, T;
+    float rho, lambda;
+};
+
+// ---------------------------------------------------------------------------------------
+// loads: the gradient rows are read exactly once, so they bypass L1 and are marked
+// evict-first in L2, which leaves the cache to the mean gradient the update reads next.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ uint4 ld_stream16(const void *p)
+{
+    uint4 r;
+    asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p));
+    return r;
+}
+
+template <int DT> struct Elem;
+template <> struct Elem<ADASCALE_F32> {
+    static constexpr int kBytes = 4, kVec = 4;
+    static __device__ __forceinline__ void unpack(const uint4 &q, float *x)
+    {
+        x[0] = __uint_as_float(q.x);
+        x[1] = __uint_as_float(q.y);
+        x[2] = __uint_as_float(q.z);
+        x[3] = __uint_as_float(q.w);
+    }
+    static __device__ __forceinline__ float load1(const void *p) { return __ldcs((const float *)p); }
+};
+template <> struct Elem<ADASCALE_BF16> {
+    static constexpr int kBytes = 2, kVec = 8;
+    // a bf16 is the upper half of an fp32: widening is a shift, exact
+    static __device__ __forceinline__ void unpack(const uint4 &q, float *x)
+    {
+        x[0] = __uint_as_float(q.x << 16);
+        x[1] = __uint_as_float(q.x & 0xffff0000u);
+        x[2] = __uint_as_float(q.y << 16);
+        x[3] = __uint_as_float(q.y & 0xffff0000u);
+        x[4] = __uint_as_float(q.z << 16);
+        x[5] = __uint_as_float(q.z & 0xffff0000u);
+        x[6] = __uint_as_float(q.w << 16);
+        x[7] = __uint_as_float(q.w & 0xffff0000u);
+    }
+    static __device__ __forceinline__ float load1(const void *p)
+    {
+        return __uint_as_float((unsigned)__ldcs((const unsigned short *)p) << 16);
+    }
+};
+
+// ---------------------------------------------------------------------------------------
+// One column vector (4 fp32 or 8 bf16 columns) of all S rows.
+//
+// Per column the S values are shifted by the first row's value c:  d_i = g_i - c.  With
+// s1 = sum d_i and s2 = sum d_i^2 the mean is c + s1/S and the summed squared deviation is
+// s2 - s1^2/S.  The shift is itself a sample, so the subtraction loses a factor of order S
+// at worst (not the |mean|^2/sigma^2 of the raw formula of App. B.3), identical rows give
+// exactly zero, and each row is consumed as it arrives: no register array of S rows.
+// B <= S rows are requested together to keep 16*B bytes per thread in flight.
+// ---------------------------------------------------------------------------------------
+template <int DT, int B>
+__device__ __forceinline__ void column_vector(const u64 *rowp, size_t boff, int S, float invS, float fS,
+                                              float *gb, float &dsum, float &nsum)
+{
+    constexpr int V = Elem<DT>::kVec;
+    float c[V], s1[V], s2[V], x[V];
+#pragma unroll
+    for (int k = 0; k < V; ++k) s1[k] = s2[k] = 0.f;
+
+    uint4 q[B];
+    // first batch: rows 0 .. B-1 (row 0 is the shift)
+#pragma unroll
+    for (int b = 0; b < B; ++b) q[b] = ld_stream16((const char *)rowp[b] + boff);
+    Elem<DT>::unpack(q[0], c);
+#pragma unroll
+    for (int b = 1; b < B; ++b) {
+        Elem<DT>::unpack(q[b], x);
+#pragma unroll
+        for (int k = 0; k < V; ++k) {
+            float d = x[k] - c[k];
+            s1[k] += d;
+            s2[k] = fmaf(d, d, s2[k]);
+        }
+    }
+    int i = B;
+    for (; i + B <= S; i += B) {
+#pragma unroll
+        for (int b = 0; b < B; ++b) q[b] = ld_stream16((const char *)rowp[i + b] + boff);
+#pragma unroll
+        for (int b = 0; b < B; ++b) {
+            Elem<DT>::unpack(q[b], x);
+#pragma unroll
+            for (int k = 0; k < V; ++k) {
+                float d = x[k] - c[k];
+                s1[k] += d;
+                s2[k] = fmaf(d, d, s2[k]);
+            }
+        }
+    }
+    for (; i < S; ++i) {
+        q[0] = ld_stream16((const char *)rowp[i] + boff);
+        Elem<DT>::unpack(q[0], x);
+#pragma unroll
+        for (int k = 0; k < V; ++k) {
+            float d = x[k] - c[k];
+            s1[k] += d;
+            s2[k] = fmaf(d, d, s2[k]);
+        }
+    }
+
+    float m[V];
+    float dacc = 0.f, nacc = 0.f;
+#pragma unroll
+    for (int k = 0; k < V; ++k) {
+        // quotient s1/S: reciprocal multiply plus one residual correction (1/S is not exact
+        // unless S is a power of two, and a biased 1/S would bias every column the same way)
+        float qk = s1[k] * invS;
+        float res = fmaf(-qk, fS, s1[k]);
+        qk = fmaf(res, invS, qk);
+        m[k] = c[k] + qk;
+        dacc += fmaf(-qk, s1[k], s2[k]);
+        nacc = fmaf(m[k], m[k], nacc);
+    }
+#pragma unroll
+    for (int k = 0; k < V; k += 4) *(float4 *)(gb + k) = make_float4(m[k], m[k + 1], m[k + 2], m[k + 3]);
+    dsum = dacc;
+    nsum = nacc;
+}
+
+// One column, any alignment, any S: plain two-pass with the residual correction of the mean.
+template <int DT>
+__device__ __forceinline__ void column_scalar(const u64 *rowp, size_t boff, int S, float fS, float *gb,
+                                              float &dsum, float &nsum)
+{
+    float sum = 0.f;
+    for (int i = 0; i < S; ++i) sum += Elem<DT>::load1((const char *)rowp[i] + boff);
+    float m0 = sum / fS;
+    float e = 0.f, qq = 0.f;
+    for (int i = 0; i < S; ++i) {
+        float d = Elem<DT>::load1((const char *)rowp[i] + boff) - m0;
+        e += d;
+        qq = fmaf(d, d, qq);
+    }
+    float corr = e / fS;
+    float m = m0 + corr;
+    *gb = m;
+    dsum = fmaf(-corr, e, qq);
+    nsum = m * m;
+}
+
+__device__ __forceinline__ double warp_sum(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Fixed-shape block sum of two doubles; result valid in thread 0.
+__device__ __forceinline__ void block_sum2(double &a, double &b, double *sa, double *sb)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    a = warp_sum(a);
+    b = warp_sum(b);
+    __syncthreads();  // scratch may still be in use by a previous call
+    if (lane == 0) {
+        sa[warp] = a;
+        sb[warp] = b;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        a = lane < kWarps ? sa[lane] : 0.0;
+        b = lane < kWarps ? sb[lane] : 0.0;
+        a = warp_sum(a);
+        b = warp_sum(b);
+    }
+}
+
+// App. B.1
+__device__ double lr_eval(const Sched &s, double t)
+{
+    if (s.kind == ADASCALE_LR_EXP) return s.eta0 * pow(s.decay, t / s.t_s1);
+    if (s.kind == ADASCALE_LR_STEP) {
+        int passed = 0;
+        for (int i = 0; i < s.n; ++i) passed += (t > s.w[i]) ? 1 : 0;
+        return s.eta0 * pow(s.decay, (double)passed);
+    }
+    return s.eta0;
+}
+
+__device__ __forceinline__ double ema(double prev, double sample, double theta, long long n)
+{
+    // plain mean of the first samples until the exponential weight takes over (App. B.3)
+    double warm = 1.0 - 1.0 / (double)n;
+    double th = theta < warm ? theta : warm;
+    return th * prev + (1.0 - th) * sample;
+}
+
+// Scalar part of the iteration: one thread, fp64, no host involvement.
+__device__ void scalar_step(DevState *st, const ScalarCfg &c, const Sched &sched, double D, double N)
+{
+    st->D = D;
+    st->N = N;
+    if (!isfinite(D) || !isfinite(N)) {  // skip the iteration, leave every average and tau alone
+        st->status = ADASCALE_STATUS_NONFINITE;
+        st->skipped += 1;
+        st->eta = 0.0;
+        return;
+    }
+    st->status = 0;
+    const double S = (double)c.S;
+    const double tau = st->tau;
+    const double t_arg = (c.flags & ADASCALE_FLAG_CONT_TAU) ? tau : floor(tau);
+    double r;
+    if (c.S == 1) {  // App. A.2: unit gain at scale one
+        st->sigma2_raw = 0.0;
+        st->mu2_raw = N;
+        r = 1.0;
+    } else {
+        double a, b, r_prior;
+        const bool ratio = (c.flags & ADASCALE_FLAG_RATIO) != 0;
+        if (ratio) {
+            // Sec. 3.4: (1/S) sum_i ||g_i||^2 = D/S + N  and ||gbar||^2
+            a = D / S + N;
+            b = N;
+            st->sigma2_raw = a;
+            st->mu2_raw = b;
+            r_prior = st->n > 0 ? (st->avg_a + c.eps) / (st->avg_b + c.eps) : 1.0;
+        } else {
+            // App. B.3: sigma^2 = D/(S-1) equals 1/(S-1) sum||g_i||^2 - S/(S-1)||gbar||^2
+            double sigma2 = D / (S - 1.0);
+            double mu2 = N - sigma2 / S;
+            st->sigma2_raw = sigma2;
+            st->mu2_raw = mu2;
+            a = sigma2 > c.eps ? sigma2 : c.eps;
+            b = mu2 > 0.0 ? mu2 : 0.0;
+            r_prior = st->n > 0 ? (st->avg_a + st->avg_b) / (st->avg_a / S + st->avg_b) : 1.0;
+        }
+        const long long n = st->n + 1;
+        const double na = ema(st->avg_a, a, c.theta, n);
+        const double nb = ema(st->avg_b, b, c.theta, n);
+        st->n = n;
+        st->avg_a = na;
+        st->avg_b = nb;
+        if (c.flags & ADASCALE_FLAG_LAGGED)
+            r = r_prior;
+        else
+            r = ratio ? (na + c.eps) / (nb + c.eps) : (na + nb) / (na / S + nb);  // Eq. 3
+    }
+    const double lr = lr_eval(sched, t_arg);
+    st->r = r;
+    st->lr = lr;
+    st->eta = r * lr;     // Sec. 3.2
+    st->tau = tau + r;
+    st->t += 1;
+}
+
+template <int DT, int B>
+__global__ void __launch_bounds__(kThreads) k_reduce(const __grid_constant__ ReduceArgs a)
+{
+    extern __shared__ u64 rowp[];
+    __shared__ double sa[kWarps], sb[kWarps];
+    __shared__ bool is_last;
+
+    constexpr int V = Elem<DT>::kVec;
+    constexpr int E = Elem<DT>::kBytes;
+    const int tid = threadIdx.x;
+    const Chunk ch = a.chunks[blockIdx.x];
+    for (int i = tid; i < a.S; i += kThreads)
+        rowp[i] = a.gptr[(size_t)i * a.T + ch.tensor] + (u64)ch.off * E;
+    __syncthreads();
+
+    float *gb = a.gbar + ch.goff;
+    double accD = 0.0, accN = 0.0;
+    int first_scalar = 0;
+    if (a.gflags[ch.tensor] & 1u) {
+        const int nv = ch.len / V;
+        for (int v = tid; v < nv; v += kThreads) {
+            float d, n;
+            column_vector<DT, B>(rowp, (size_t)v * 16, a.S, a.invS, a.fS, gb + (size_t)v * V, d, n);
+            accD += (double)d;
+            accN += (double)n;
+        }
+        first_scalar = nv * V;
+    }
+    for (int e = first_scalar + tid; e < ch.len; e += kThreads) {
+        float d, n;
+        column_scalar<DT>(rowp, (size_t)e * E, a.S, a.fS, gb + e, d, n);
+        accD += (double)d;
+        accN += (double)n;
+    }
+
+    block_sum2(accD, accN, sa, sb);
+    if (tid == 0) {
+        a.partials[blockIdx.x] = make_double2(accD, accN);
+        __threadfence();
+        const unsigned tk = atomicAdd(a.ticket, 1u);
+        is_last = (tk == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+
+    // Second stage, fixed order: thread j adds partials j, j+256, ... in index order, then the
+    // same block tree.  The result depends on the chunk table only, not on block scheduling.
+    __threadfence();
+    double d = 0.0, n = 0.0;
+    for (int i = tid; i < (int)gridDim.x; i += kThreads) {
+        const double2 p = __ldcg(&a.partials[i]);
+        d += p.x;
+        n += p.y;
+    }
+    block_sum2(d, n, sa, sb);
+    if (tid == 0) {
+        scalar_step(a.st, a.sc, a.sched, d, n);
+        *a.ticket = 0u;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) k_update(const __grid_constant__ UpdateArgs a)
+{
+    if (a.st->status & ADASCALE_STATUS_NONFINITE) return;
+    const float eta = (float)a.st->eta;
+    // newest mean-gradient chunks first: they are the most likely to still sit in L2
+    const Chunk ch = a.chunks[a.n_chunks - 1 - (int)blockIdx.x];
+    float *w = (float *)a.wv[ch.tensor] + ch.off;
+    float *v = (float *)a.wv[a.T + ch.tensor] + ch.off;
+    const float *g = a.gbar + ch.goff;
+    const int tid = threadIdx.x;
+    int first_scalar = 0;
+    if (a.wflags[ch.tensor] & 1u) {
+        const int nv = ch.len >> 2;
+        for (int i = tid; i < nv; i += kThreads) {
+            const float4 gg = ((const float4 *)g)[i];
+            float4 ww = ((const float4 *)w)[i];
+            float4 vv = ((const float4 *)v)[i];
+            vv.x = fmaf(a.rho, vv.x, fmaf(a.lambda, ww.x, gg.x));
+            vv.y = fmaf(a.rho, vv.y, fmaf(a.lambda, ww.y, gg.y));
+            vv.z = fmaf(a.rho, vv.z, fmaf(a.lambda, ww.z, gg.z));
+            vv.w = fmaf(a.rho, vv.w, fmaf(a.lambda, ww.w, gg.w));
+            ww.x = fmaf(-eta, vv.x, ww.x);
+            ww.y = fmaf(-eta, vv.y, ww.y);
+            ww.z = fmaf(-eta, vv.z, ww.z);
+            ww.w = fmaf(-eta, vv.w, ww.w);
+            ((float4 *)v)[i] = vv;
+            ((float4 *)w)[i] = ww;
+        }
+        first_scalar = nv << 2;
+    }
+    for (int e = first_scalar + tid; e < ch.len; e += kThreads) {
+        const float vn = fmaf(a.rho, v[e], fmaf(a.lambda, w[e], g[e]));
+        v[e] = vn;
+        w[e] = fmaf(-eta, vn, w[e]);
+    }
+}
+
+// ---- bandwidth probes -------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads) k_probe_read(const uint4 *a, long long n, unsigned *sink)
+{
+    unsigned acc = 0;
+    for (long long i = (long long)blockIdx.x * kThreads + threadIdx.x; i < n; i += (long long)gridDim.x * kThreads) {
+        const uint4 q = ld_stream16(a + i);
+        acc ^= q.x ^ q.y ^ q.z ^ q.w;
+    }
+    if (acc == 0x9e3779b9u) *sink = acc;  // keeps the loads alive, practically never taken
+}
+__global__ void __launch_bounds__(kThreads) k_probe_copy(const uint4 *a, uint4 *b, long long n)
+{
+    for (long long i = (long long)blockIdx.x * kThreads + threadIdx.x; i < n; i += (long long)gridDim.x * kThreads)
+        b[i] = ld_stream16(a + i);
+}
+__global__ void __launch_bounds__(kThreads) k_probe_rmw(float4 *a, const float4 *b, long long n)
+{
+    for (long long i = (long long)blockIdx.x * kThreads + threadIdx.x; i < n; i += (long long)gridDim.x * kThreads) {
+        float4 x = a[i];
+        const float4 y = b[i];
+        x.x += y.x;
+        x.y += y.y;
+        x.z += y.z;
+        x.w += y.w;
+        a[i] = x;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------
+
+// A table of pointers (plus per-tensor flags) mirrored on the host and uploaded only when
+// it changes, through a small ring of pinned slots so that an upload still in flight is
+// never overwritten.
+struct PtrTable {
+    std::vector<u64> mirror;   // last uploaded contents (pointers then flags, 8-byte units)
+    u64 *dev = nullptr;
+    u64 *pinned[kRing] = {nullptr, nullptr, nullptr, nullptr};
+    cudaEvent_t ev[kRing] = {nullptr, nullptr, nullptr, nullptr};
+    bool used[kRing] = {false, false, false, false};
+    int next = 0;
+    size_t words = 0;
+    bool valid = false;
+};
+
+struct StateBlob {  // ADASCALE_STATE_BYTES
+    unsigned magic, version;
+    int S;
+    unsigned flags;
+    double tau, avg_a, avg_b;
+    long long n, t, skipped;
+    double r, eta, lr;
+    double pad[5];
+};
+static_assert(sizeof(StateBlob) == ADASCALE_STATE_BYTES, "state blob size");
+constexpr unsigned kMagic = 0x41645363u;  // "AdSc"
+
+}  // namespace
+
+struct adascale_ctx {
+    int device = 0;
+    int S = 1, max_S = 1, T = 0, dtype = 0;
+    double rho = 0, lambda = 0, eps = 1e-6, theta_cfg = -1;
+    unsigned flags = 0;
+    std::vector<long long> numel;
+    std::vector<long long> goff;
+    long long P = 0, gbar_elems = 0;
+    int n_chunks = 0;
+    Chunk *d_chunks = nullptr;
+    float *d_gbar = nullptr;
+    double2 *d_partials = nullptr;
+    unsigned *d_ticket = nullptr;
+    DevState *d_state = nullptr;
+    PtrTable tg, tw;
+    DevState *h_snap = nullptr;      // pinned, 2 slots
+    cudaEvent_t ev_snap = nullptr;
+    bool snap_inflight = false;
+    DevState latest{};
+    cudaStream_t last_stream = nullptr;
+    bool reduced = false;
+    long long launches = 0;
+    // host-gradient staging (adascale_step_host)
+    void *d_stage = nullptr;
+    std::vector<const void *> stage_ptrs;
+    std::string err;
+};
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard()
+    {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+adascale_status cuda_fail(adascale_ctx *c, cudaError_t e, const char *what)
+{
+    if (c) {
+        c->err = what;
+        c->err += ": ";
+        c->err += cudaGetErrorString(e);
+    }
+    cudaGetLastError();  // a non-sticky error must not leak into the caller's next CUDA call
+    return ADASCALE_ERR_CUDA;
+}
+
+#define CU(call)                                                    \
+    do {                                                            \
+        cudaError_t e_ = (call);                                    \
+        if (e_ != cudaSuccess) return cuda_fail(ctx, e_, #call);    \
+    } while (0)
+
+double resolve_theta(const adascale_ctx *c)
+{
+    if (c->theta_cfg >= 0.0) return c->theta_cfg;
+    const double th = 1.0 - (double)c->S / 1000.0;  // Sec. 3.4: theta = max{1 - S/1000, 0}
+    return th > 0.0 ? th : 0.0;
+}
+
+adascale_status table_alloc(adascale_ctx *ctx, PtrTable &t, size_t words)
+{
+    t.words = words;
+    t.mirror.assign(words, 0);
+    CU(cudaMalloc(&t.dev, words * sizeof(u64)));
+    for (int i = 0; i < kRing; ++i) {
+        CU(cudaMallocHost(&t.pinned[i], words * sizeof(u64)));
+        CU(cudaEventCreateWithFlags(&t.ev[i], cudaEventDisableTiming));
+    }
+    return ADASCALE_OK;
+}
+
+void table_free(PtrTable &t)
+{
+    if (t.dev) cudaFree(t.dev);
+    for (int i = 0; i < kRing; ++i) {
+        if (t.pinned[i]) cudaFreeHost(t.pinned[i]);
+        if (t.ev[i]) cudaEventDestroy(t.ev[i]);
+    }
+    t = PtrTable();
+}
+
+// Uploads `fresh` (t.words entries) if it differs from what the device already holds.
+adascale_status table_sync(adascale_ctx *ctx, PtrTable &t, const std::vector<u64> &fresh, cudaStream_t s)
+{
+    if (t.valid && std::memcmp(fresh.data(), t.mirror.data(), t.words * sizeof(u64)) == 0) return ADASCALE_OK;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    CU(cudaStreamIsCapturing(s, &cap));
+    if (cap != cudaStreamCaptureStatusNone) {
+        ctx->err = "pointer table changed inside a stream capture";
+        return ADASCALE_ERR_STATE;
+    }
+    const int slot = t.next;
+    t.next = (t.next + 1) % kRing;
+    if (t.used[slot]) CU(cudaEventSynchronize(t.ev[slot]));
+    std::memcpy(t.pinned[slot], fresh.data(), t.words * sizeof(u64));
+    CU(cudaMemcpyAsync(t.dev, t.pinned[slot], t.words * sizeof(u64), cudaMemcpyHostToDevice, s));
+    CU(cudaEventRecord(t.ev[slot], s));
+    t.used[slot] = true;
+    t.mirror = fresh;
+    t.valid = true;
+    return ADASCALE_OK;
+}
+
+template <int DT>
+cudaError_t launch_reduce(int B, const ReduceArgs &a, size_t smem, cudaStream_t s)
+{
+    const dim3 grid(a.n_chunks), block(kThreads);
+    switch (B) {
+    case 1: k_reduce<DT, 1><<<grid, block, smem, s>>>(a); break;
+    case 2: k_reduce<DT, 2><<<grid, block, smem, s>>>(a); break;
+    case 4: k_reduce<DT, 4><<<grid, block, smem, s>>>(a); break;
+    default: k_reduce<DT, 8><<<grid, block, smem, s>>>(a); break;
+    }
+    return cudaGetLastError();
+}
+
+int batch_for(int S) { return S >= 8 ? 8 : S >= 4 ? 4 : S >= 2 ? 2 : 1; }
+
+bool valid_sched(const adascale_lr_schedule *s)
+{
+    if (!s) return false;
+    if (s->kind < ADASCALE_LR_CONST || s->kind > ADASCALE_LR_STEP) return false;
+    if (!(s->eta0 > 0.0)) return false;
+    if (s->kind != ADASCALE_LR_CONST && !(s->decay > 0.0)) return false;
+    if (s->kind == ADASCALE_LR_EXP && !(s->t_s1 > 0.0)) return false;
+    if (s->kind == ADASCALE_LR_STEP && (s->n_milestones < 0 || s->n_milestones > ADASCALE_MAX_MILESTONES)) return false;
+    return true;
+}
+
+adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const adascale_lr_schedule *sched,
+                          cudaStream_t s)
+{
+    const int S = ctx->S, T = ctx->T;
+    const size_t esz = ctx->dtype == ADASCALE_BF16 ? 2 : 4;
+    std::vector<u64> fresh(ctx->tg.words, 0);
+    unsigned *flags = reinterpret_cast<unsigned *>(fresh.data() + (size_t)ctx->max_S * T);
+    for (int k = 0; k < T; ++k) {
+        unsigned aligned = 1u;
+        for (int i = 0; i < S; ++i) {
+            const u64 p = (u64)(uintptr_t)grads[(size_t)i * T + k];
+            if (ctx->numel[k] > 0) {
+                if (p == 0) return ADASCALE_ERR_INVALID_ARG;
+                if (p % esz) return ADASCALE_ERR_ALIGNMENT;
+                if (p % 16) aligned = 0u;
+            }
+            fresh[(size_t)i * T + k] = p;
+        }
+        flags[k] = aligned;
+    }
+    adascale_status st = table_sync(ctx, ctx->tg, fresh, s);
+    if (st != ADASCALE_OK) return st;
+    if (ctx->n_chunks == 0) return ADASCALE_OK;
+
+    ReduceArgs a;
+    a.chunks = ctx->d_chunks;
+    a.gptr = ctx->tg.dev;
+    a.gflags = reinterpret_cast<const unsigned *>(ctx->tg.dev + (size_t)ctx->max_S * T);
+    a.gbar = ctx->d_gbar;
+    a.partials = ctx->d_partials;
+    a.ticket = ctx->d_ticket;
+    a.st = ctx->d_state;
+    a.n_chunks = ctx->n_chunks;
+    a.S = S;
+    a.T = T;
+    a.fS = (float)S;
+    a.invS = 1.0f / (float)S;
+    a.sc.eps = ctx->eps;
+    a.sc.theta = resolve_theta(ctx);
+    a.sc.flags = ctx->flags;
+    a.sc.S = S;
+    a.sched.kind = sched->kind;
+    a.sched.n = sched->kind == ADASCALE_LR_STEP ? sched->n_milestones : 0;
+    a.sched.eta0 = sched->eta0;
+    a.sched.decay = sched->decay;
+    a.sched.t_s1 = sched->t_s1;
+    for (int i = 0; i < ADASCALE_MAX_MILESTONES; ++i) a.sched.w[i] = sched->milestones[i];
+
+    const size_t smem = (size_t)S * sizeof(u64);
+    const int B = batch_for(S);
+    cudaError_t e = ctx->dtype == ADASCALE_BF16 ? launch_reduce<ADASCALE_BF16>(B, a, smem, s)
+                                                : launch_reduce<ADASCALE_F32>(B, a, smem, s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "launch of the reduce kernel");
+    ctx->launches += 1;
+    ctx->reduced = true;
+    ctx->last_stream = s;
+    return ADASCALE_OK;
+}
+
+adascale_status do_update(adascale_ctx *ctx, void *const *params, void *const *momentum, cudaStream_t s)
+{
+    const int T = ctx->T;
+    std::vector<u64> fresh(ctx->tw.words, 0);
+    unsigned *flags = reinterpret_cast<unsigned *>(fresh.data() + (size_t)2 * T);
+    for (int k = 0; k < T; ++k) {
+        const u64 pw = (u64)(uintptr_t)params[k], pv = (u64)(uintptr_t)momentum[k];
+        if (ctx->numel[k] > 0) {
+            if (!pw || !pv) return ADASCALE_ERR_INVALID_ARG;
+            if ((pw % 4) || (pv % 4)) return ADASCALE_ERR_ALIGNMENT;
+        }
+        fresh[k] = pw;
+        fresh[(size_t)T + k] = pv;
+        flags[k] = ((pw % 16) == 0 && (pv % 16) == 0) ? 1u : 0u;
+    }
+    adascale_status st = table_sync(ctx, ctx->tw, fresh, s);
+    if (st != ADASCALE_OK) return st;
+    if (ctx->n_chunks == 0) return ADASCALE_OK;
+
+    UpdateArgs a;
+    a.chunks = ctx->d_chunks;
+    a.wv = ctx->tw.dev;
+    a.wflags = reinterpret_cast<const unsigned *>(ctx->tw.dev + (size_t)2 * T);
+    a.gbar = ctx->d_gbar;
+    a.st = ctx->d_state;
+    a.n_chunks = ctx->n_chunks;
+    a.T = T;
+    a.rho = (float)ctx->rho;
+    a.lambda = (float)ctx->lambda;
+    k_update<<<dim3(ctx->n_chunks), dim3(kThreads), 0, s>>>(a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "launch of the update kernel");
+    ctx->launches += 1;
+    ctx->last_stream = s;
+    return ADASCALE_OK;
+}
+
+void fill_stats(const adascale_ctx *ctx, const DevState &d, adascale_stats *o)
+{
+    std::memset(o, 0, sizeof *o);
+    o->r = d.r;
+    o->tau = d.tau;
+    o->eta = d.eta;
+    o->lr = d.lr;
+    o->sigma2_raw = d.sigma2_raw;
+    o->mu2_raw = d.mu2_raw;
+    o->sigma2_avg = d.avg_a;
+    o->mu2_avg = d.avg_b;
+    o->gbar_sqnorm = d.N;
+    o->dev_sqsum = d.D;
+    o->t = d.t;
+    o->n_samples = d.n;
+    o->skipped = d.skipped;
+    o->status_bits = d.status;
+    (void)ctx;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *adascale_strerror(adascale_status s)
+{
+    switch (s) {
+    case ADASCALE_OK: return "ok";
+    case ADASCALE_ERR_INVALID_ARG: return "invalid argument";
+    case ADASCALE_ERR_ALIGNMENT: return "pointer not aligned to its element size";
+    case ADASCALE_ERR_CUDA: return "CUDA runtime error";
+    case ADASCALE_ERR_STATE: return "call not allowed in the current state";
+    case ADASCALE_ERR_TOO_LARGE: return "size beyond the documented maximum";
+    }
+    return "unknown status";
+}
+
+const char *adascale_last_error(const adascale_ctx *ctx) { return ctx ? ctx->err.c_str() : ""; }
+
+int64_t adascale_launch_count(const adascale_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+adascale_status adascale_init(const adascale_config *cfg, adascale_ctx **out)
+{
+    if (!cfg || !out) return ADASCALE_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (cfg->S < 1 || cfg->n_tensors < 1 || !cfg->numel) return ADASCALE_ERR_INVALID_ARG;
+    const int max_S = cfg->max_S > 0 ? cfg->max_S : cfg->S;
+    if (max_S < cfg->S) return ADASCALE_ERR_INVALID_ARG;
+    if (max_S > kMaxS) return ADASCALE_ERR_TOO_LARGE;
+    if (cfg->grad_dtype != ADASCALE_F32 && cfg->grad_dtype != ADASCALE_BF16) return ADASCALE_ERR_INVALID_ARG;
+    if (!(cfg->theta < 1.0) || !(cfg->eps >= 0.0) || cfg->device < 0) return ADASCALE_ERR_INVALID_ARG;
+    if (!std::isfinite(cfg->momentum) || !std::isfinite(cfg->weight_decay)) return ADASCALE_ERR_INVALID_ARG;
+    if (cfg->flags & ~(ADASCALE_FLAG_LAGGED | ADASCALE_FLAG_CONT_TAU | ADASCALE_FLAG_RATIO))
+        return ADASCALE_ERR_INVALID_ARG;
+    for (int k = 0; k < cfg->n_tensors; ++k)
+        if (cfg->numel[k] < 0) return ADASCALE_ERR_INVALID_ARG;
+
+    adascale_ctx *ctx = new (std::nothrow) adascale_ctx();
+    if (!ctx) return ADASCALE_ERR_INVALID_ARG;
+    ctx->device = cfg->device;
+    ctx->S = cfg->S;
+    ctx->max_S = max_S;
+    ctx->T = cfg->n_tensors;
+    ctx->dtype = cfg->grad_dtype;
+    ctx->rho = cfg->momentum;
+    ctx->lambda = cfg->weight_decay;
+    ctx->eps = cfg->eps;
+    ctx->theta_cfg = cfg->theta;
+    ctx->flags = cfg->flags;
+    ctx->numel.assign(cfg->numel, cfg->numel + cfg->n_tensors);
+
+    // chunk table: every tensor is cut into blocks of kChunk elements; chunk boundaries are
+    // multiples of 8 elements so a 16-byte aligned tensor stays 16-byte aligned in every chunk
+    const int chunk = ctx->dtype == ADASCALE_BF16 ? kChunkBF16 : kChunkF32;
+    std::vector<Chunk> chunks;
+    long long g = 0;
+    for (int k = 0; k < ctx->T; ++k) {
+        ctx->goff.push_back(g);
+        const long long n = ctx->numel[k];
+        for (long long o = 0; o < n; o += chunk) {
+            Chunk c;
+            c.off = o;
+            c.goff = g + o;
+            c.tensor = k;
+            c.len = (int)((n - o) < chunk ? (n - o) : chunk);
+            chunks.push_back(c);
+        }
+        ctx->P += n;
+        g += (n + kGbarAlign - 1) / kGbarAlign * kGbarAlign;
+    }
+    ctx->gbar_elems = g;
+    if (chunks.size() > 0x7fffffffull) {
+        delete ctx;
+        return ADASCALE_ERR_TOO_LARGE;
+    }
+    ctx->n_chunks = (int)chunks.size();
+
+    DeviceGuard guard(ctx->device);
+    adascale_status rc = ADASCALE_OK;
+    auto body = [&]() -> adascale_status {
+        if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
+        const size_t nc = chunks.empty() ? 1 : chunks.size();
+        CU(cudaMalloc(&ctx->d_chunks, nc * sizeof(Chunk)));
+        if (!chunks.empty())
+            CU(cudaMemcpy(ctx->d_chunks, chunks.data(), chunks.size() * sizeof(Chunk), cudaMemcpyHostToDevice));
+        CU(cudaMalloc(&ctx->d_gbar, (size_t)(g > 0 ? g : 1) * sizeof(float)));
+        CU(cudaMemset(ctx->d_gbar, 0, (size_t)(g > 0 ? g : 1) * sizeof(float)));
+        CU(cudaMalloc(&ctx->d_partials, nc * sizeof(double2)));
+        CU(cudaMalloc(&ctx->d_ticket, sizeof(unsigned)));
+        CU(cudaMemset(ctx->d_ticket, 0, sizeof(unsigned)));
+        CU(cudaMalloc(&ctx->d_state, sizeof(DevState)));
+        CU(cudaMemset(ctx->d_state, 0, sizeof(DevState)));
+        const size_t T = (size_t)ctx->T;
+        adascale_status s1 = table_alloc(ctx, ctx->tg, (size_t)ctx->max_S * T + (T + 1) / 2);
+        if (s1 != ADASCALE_OK) return s1;
+        s1 = table_alloc(ctx, ctx->tw, 2 * T + (T + 1) / 2);
+        if (s1 != ADASCALE_OK) return s1;
+        CU(cudaMallocHost(&ctx->h_snap, sizeof(DevState)));
+        std::memset(ctx->h_snap, 0, sizeof(DevState));
+        CU(cudaEventCreateWithFlags(&ctx->ev_snap, cudaEventDisableTiming));
+        // dynamic shared memory of the reduce kernel: S row pointers (32 KB at the maximum S)
+        return ADASCALE_OK;
+    };
+    rc = body();
+    if (rc != ADASCALE_OK) {
+        adascale_destroy(ctx);
+        return rc;
+    }
+    *out = ctx;
+    return ADASCALE_OK;
+}
+
+adascale_status adascale_destroy(adascale_ctx *ctx)
+{
+    if (!ctx) return ADASCALE_OK;
+    DeviceGuard guard(ctx->device);
+    if (guard.ok) {
+        cudaDeviceSynchronize();
+        cudaFree(ctx->d_chunks);
+        cudaFree(ctx->d_gbar);
+        cudaFree(ctx->d_partials);
+        cudaFree(ctx->d_ticket);
+        cudaFree(ctx->d_state);
+        cudaFree(ctx->d_stage);
+        table_free(ctx->tg);
+        table_free(ctx->tw);
+        if (ctx->h_snap) cudaFreeHost(ctx->h_snap);
+        if (ctx->ev_snap) cudaEventDestroy(ctx->ev_snap);
+        cudaGetLastError();
+    }
+    delete ctx;
+    return ADASCALE_OK;
+}
+
+adascale_status adascale_reduce(adascale_ctx *ctx, const void *const *grads, const adascale_lr_schedule *sched,
+                                void *cuda_stream)
+{
+    if (!ctx || !grads || !valid_sched(sched)) return ADASCALE_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
+    return do_reduce(ctx, grads, sched, (cudaStream_t)cuda_stream);
+}
+
+adascale_status adascale_update(adascale_ctx *ctx, void *const *params, void *const *momentum, void *cuda_stream)
+{
+    if (!ctx || !params || !momentum) return ADASCALE_ERR_INVALID_ARG;
+    if (!ctx->reduced) return ADASCALE_ERR_STATE;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
+    return do_update(ctx, params, momentum, (cudaStream_t)cuda_stream);
+}
+
+adascale_status adascale_step(adascale_ctx *ctx, const void *const *grads, void *const *params,
+                              void *const *momentum, const adascale_lr_schedule *sched, void *cuda_stream)
+{
+    if (!ctx || !grads || !params || !momentum || !valid_sched(sched)) return ADASCALE_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
+    // validate the update's pointers before anything is enqueued
+    for (int k = 0; k < ctx->T; ++k) {
+        if (ctx->numel[k] > 0) {
+            if (!params[k] || !momentum[k]) return ADASCALE_ERR_INVALID_ARG;
+            if (((uintptr_t)params[k] % 4) || ((uintptr_t)momentum[k] % 4)) return ADASCALE_ERR_ALIGNMENT;
+        }
+    }
+    adascale_status st = do_reduce(ctx, grads, sched, (cudaStream_t)cuda_stream);
+    if (st != ADASCALE_OK) return st;
+    return do_update(ctx, params, momentum, (cudaStream_t)cuda_stream);
+}
+
+adascale_status adascale_get_gain_tau(adascale_ctx *ctx, adascale_stats *out, int blocking)
+{
+    if (!ctx || !out) return ADASCALE_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
+    cudaStream_t s = ctx->last_stream;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    CU(cudaStreamIsCapturing(s, &cap));
+    if (cap != cudaStreamCaptureStatusNone) return ADASCALE_ERR_STATE;
+    if (ctx->snap_inflight) {
+        if (blocking) {
+            CU(cudaEventSynchronize(ctx->ev_snap));
+            ctx->latest = *ctx->h_snap;
+            ctx->snap_inflight = false;
+        } else {
+            cudaError_t q = cudaEventQuery(ctx->ev_snap);
+            if (q == cudaSuccess) {
+                ctx->latest = *ctx->h_snap;
+                ctx->snap_inflight = false;
+            } else if (q != cudaErrorNotReady) {
+                return cuda_fail(ctx, q, "cudaEventQuery");
+            }
+        }
+    }
+    if (!ctx->snap_inflight) {
+        CU(cudaMemcpyAsync(ctx->h_snap, ctx->d_state, sizeof(DevState), cudaMemcpyDeviceToHost, s));
+        CU(cudaEventRecord(ctx->ev_snap, s));
+        ctx->snap_inflight = true;
+        if (blocking) {
+            CU(cudaEventSynchronize(ctx->ev_snap));
+            ctx->latest = *ctx->h_snap;
+            ctx->snap_inflight = false;
+        }
+    }
+    fill_stats(ctx, ctx->latest, out);
+    return ADASCALE_OK;
+}
+
+adascale_status adascale_mean_grad(adascale_ctx *ctx, const void **gbar)
+{
+    if (!ctx || !gbar) return ADASCALE_ERR_INVALID_ARG;
+    for (int k = 0; k < ctx->T; ++k) gbar[k] = ctx->d_gbar + ctx->goff[k];
+    return ADASCALE_OK;
+}
+
+adascale_status adascale_set_scale(adascale_ctx *ctx, int32_t S)
+{
+    if (!ctx || S < 1) return ADASCALE_ERR_INVALID_ARG;
+    if (S > ctx->max_S) return ADASCALE_ERR_TOO_LARGE;
+    if (S != ctx->S) {
+        ctx->S = S;
+        ctx->tg.valid = false;
+    }
+    return ADASCALE_OK;
+}
+
+adascale_status adascale_get_state(adascale_ctx *ctx, void *buf)
+{
+    if (!ctx || !buf) return ADASCALE_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
+    DevState d;
+    CU(cudaStreamSynchronize(ctx->last_stream));
+    CU(cudaMemcpy(&d, ctx->d_state, sizeof d, cudaMemcpyDeviceToHost));
+    StateBlob b;
+    std::memset(&b, 0, sizeof b);
+    b.magic = kMagic;
+    b.version = 1;
+    b.S = ctx->S;
+    b.flags = ctx->flags;
+    b.tau = d.tau;
+    b.avg_a = d.avg_a;
+    b.avg_b = d.avg_b;
+    b.n = d.n;
+    b.t = d.t;
+    b.skipped = d.skipped;
+    b.r = d.r;
+    b.eta = d.eta;
+    b.lr = d.lr;
+    std::memcpy(buf, &b, sizeof b);
+    return ADASCALE_OK;
+}
+
+adascale_status adascale_set_state(adascale_ctx *ctx, const void *buf)
+{
+    if (!ctx || !buf) return ADASCALE_ERR_INVALID_ARG;
+    StateBlob b;
+    std::memcpy(&b, buf, sizeof b);
+    if (b.magic != kMagic || b.version != 1) return ADASCALE_ERR_INVALID_ARG;
+    if (b.S < 1 || b.S > ctx->max_S) return ADASCALE_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
+    DevState d;
+    std::memset(&d, 0, sizeof d);
+    d.tau = b.tau;
+    d.avg_a = b.avg_a;
+    d.avg_b = b.avg_b;
+    d.n = b.n;
+    d.t = b.t;
+    d.skipped = b.skipped;
+    d.r = b.r;
+    d.eta = b.eta;
+    d.lr = b.lr;
+    CU(cudaStreamSynchronize(ctx->last_stream));
+    CU(cudaMemcpy(ctx->d_state, &d, sizeof d, cudaMemcpyHostToDevice));
+    if (b.S != ctx->S) {
+        ctx->S = b.S;
+        ctx->tg.valid = false;
+    }
+    ctx->reduced = false;
+    return ADASCALE_OK;
+}
+
+adascale_status adascale_step_host(adascale_ctx *ctx, const void *const *grads, void *const *params,
+                                   void *const *momentum, const adascale_lr_schedule *sched,
+                                   adascale_stats *out, void *cuda_stream)
+{
+    if (!ctx || !grads || !params || !momentum || !valid_sched(sched)) return ADASCALE_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const size_t esz = ctx->dtype == ADASCALE_BF16 ? 2 : 4;
+    const int S = ctx->S, T = ctx->T;
+    if (!ctx->d_stage) {
+        CU(cudaMalloc(&ctx->d_stage, (size_t)ctx->max_S * (size_t)(ctx->gbar_elems > 0 ? ctx->gbar_elems : 1) * esz));
+    }
+    ctx->stage_ptrs.assign((size_t)S * T, nullptr);
+    for (int i = 0; i < S; ++i)
+        for (int k = 0; k < T; ++k)
+            if (ctx->numel[k] > 0 && !grads[(size_t)i * T + k]) return ADASCALE_ERR_INVALID_ARG;
+    for (int i = 0; i < S; ++i) {
+        char *row = (char *)ctx->d_stage + (size_t)i * ctx->gbar_elems * esz;
+        // tensors that continue each other in host memory and in the staging row travel as one copy
+        const char *run_src = nullptr;
+        char *run_dst = nullptr;
+        size_t run_bytes = 0;
+        for (int k = 0; k < T; ++k) {
+            const char *src = (const char *)grads[(size_t)i * T + k];
+            char *dst = row + (size_t)ctx->goff[k] * esz;
+            ctx->stage_ptrs[(size_t)i * T + k] = dst;
+            const size_t bytes = (size_t)ctx->numel[k] * esz;
+            if (bytes == 0) continue;
+            if (run_bytes && src == run_src + run_bytes && dst == run_dst + run_bytes) {
+                run_bytes += bytes;
+                continue;
+            }
+            if (run_bytes) CU(cudaMemcpyAsync(run_dst, run_src, run_bytes, cudaMemcpyHostToDevice, s));
+            run_src = src;
+            run_dst = dst;
+            run_bytes = bytes;
+        }
+        if (run_bytes) CU(cudaMemcpyAsync(run_dst, run_src, run_bytes, cudaMemcpyHostToDevice, s));
+    }
+    adascale_status st = adascale_step(ctx, ctx->stage_ptrs.data(), params, momentum, sched, cuda_stream);
+    if (st != ADASCALE_OK) return st;
+    adascale_stats tmp;
+    st = adascale_get_gain_tau(ctx, out ? out : &tmp, 1);
+    if (st != ADASCALE_OK) return st;
+    CU(cudaStreamSynchronize(s));
+    return ADASCALE_OK;
+}
+
+adascale_status adascale_stream_probe(int32_t kind, void *a, void *b, int64_t n_bytes, void *cuda_stream)
+{
+    adascale_ctx *ctx = nullptr;
+    if (!a || n_bytes < 16 || (n_bytes % 16) || ((uintptr_t)a % 16)) return ADASCALE_ERR_INVALID_ARG;
+    if (kind < 0 || kind > 2) return ADASCALE_ERR_INVALID_ARG;
+    if (kind != 0 && (!b || ((uintptr_t)b % 16))) return ADASCALE_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const long long n = n_bytes / 16;
+    int dev = 0, sms = 0;
+    CU(cudaGetDevice(&dev));
+    CU(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    long long blocks = (n + kThreads - 1) / kThreads;
+    const long long cap = (long long)sms * 32;
+    if (blocks > cap) blocks = cap;
+    if (kind == 0) {
+        if (!b) return ADASCALE_ERR_INVALID_ARG;  // 4-byte sink that keeps the loads alive
+        k_probe_read<<<(unsigned)blocks, kThreads, 0, s>>>((const uint4 *)a, n, (unsigned *)b);
+    } else if (kind == 1) {
+        k_probe_copy<<<(unsigned)blocks, kThreads, 0, s>>>((const uint4 *)a, (uint4 *)b, n);
+    } else {
+        k_probe_rmw<<<(unsigned)blocks, kThreads, 0, s>>>((float4 *)a, (const float4 *)b, n);
+    }
+    CU(cudaGetLastError());
+    return ADASCALE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,333 @@
+"""Parity of the CUDA library (through its C ABI) with the CPU oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+if not torch.cuda.is_available():
+    pytest.skip("needs a CUDA device", allow_module_level=True)
+
+import _harness as H  # noqa: E402
+from paper_2007_05105_b200 import binding as B  # noqa: E402
+from paper_2007_05105_b200 import synthetic  # noqa: E402
+
+DEV = torch.device("cuda:0")
+RAGGED = [1, 3, 4, 5, 7, 8, 9, 1023, 1025, 2048, 2049, 4097, 10000]
+
+
+def _gen(seed):
+    g = torch.Generator(device=DEV)
+    g.manual_seed(seed)
+    return g
+
+
+def _make_rows(numels, S, dtype, gen, k=3.0, mean_std=0.1, misalign=0):
+    """Separate allocations per (row, tensor); `misalign` shifts every view by that many elements."""
+    mean = [torch.empty(n, device=DEV).normal_(0, mean_std, generator=gen) for n in numels]
+    rows = []
+    for _ in range(S):
+        row = []
+        for n, m in zip(numels, mean):
+            buf = torch.empty(n + misalign, device=DEV, dtype=torch.float32).normal_(0, 1, generator=gen)
+            full = torch.empty(n + misalign, device=DEV, dtype=dtype)
+            full[misalign:] = (m + k * mean_std * buf[misalign:]).to(dtype)
+            row.append(full[misalign:])
+        rows.append(row)
+    return rows
+
+
+def _params(numels, gen, misalign=0):
+    w = [torch.empty(n + misalign, device=DEV).normal_(0, 1, generator=gen)[misalign:] for n in numels]
+    v = [torch.empty(n + misalign, device=DEV).normal_(0, 0.1, generator=gen)[misalign:] for n in numels]
+    return w, v
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("S", [1, 2, 3, 4, 5, 7, 8, 9, 16, 17, 32, 33, 40])
+def test_ragged_tensor_list(S, dtype):
+    gen = _gen(1000 + S)
+    name = "bf16" if dtype == torch.bfloat16 else "f32"
+    pair = H.Pair(RAGGED, S, name, momentum=0.9, weight_decay=1e-3, lr={"kind": "const", "eta0": 0.05})
+    w, v = _params(RAGGED, gen)
+    pair.attach(w, v)
+    for step in range(3):
+        rows = _make_rows(RAGGED, S, dtype, gen, k=[0.5, 3.0, 10.0][step])
+        pair.step(rows, "S=%d %s step %d" % (S, name, step))
+    pair.close()
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("misalign", [1, 2, 3])
+def test_misaligned_pointers_take_the_scalar_path(misalign, dtype):
+    gen = _gen(77 + misalign)
+    numels = [5, 64, 1000, 4099]
+    name = "bf16" if dtype == torch.bfloat16 else "f32"
+    pair = H.Pair(numels, 5, name, momentum=0.5, weight_decay=0.01)
+    w, v = _params(numels, gen, misalign)
+    pair.attach(w, v)
+    for step in range(2):
+        pair.step(_make_rows(numels, 5, dtype, gen, misalign=misalign), "misalign %d step %d" % (misalign, step))
+    pair.close()
+
+
+def test_empty_tensors_are_skipped():
+    gen = _gen(5)
+    numels = [0, 17, 0, 256, 0]
+    pair = H.Pair(numels, 4)
+    w, v = _params(numels, gen)
+    pair.attach(w, v)
+    pair.step(_make_rows(numels, 4, torch.float32, gen), "empty")
+    pair.close()
+
+
+def test_identical_rows_zero_variance():
+    gen = _gen(6)
+    numels = [4096 + 5, 333]
+    for S in (2, 3, 8, 32):
+        base = [torch.empty(n, device=DEV).normal_(0, 1, generator=gen) for n in numels]
+        rows = [[b.clone() for b in base] for _ in range(S)]
+        pair = H.Pair(numels, S, theta=0.0)
+        w, v = _params(numels, gen)
+        pair.attach(w, v)
+        st, ost = pair.step(rows, "identical S=%d" % S)
+        assert st.dev_sqsum == 0.0 and st.sigma2_raw == 0.0
+        assert abs(st.r - 1.0) < 1e-6
+        pair.close()
+
+
+def test_extreme_conditioning_k30_and_k0():
+    """mu^2 is ~1/113 of ||gbar||^2 at k = 30, S = 8: the worst case for the subtraction."""
+    gen = _gen(8)
+    numels = [300000, 77]
+    for k in (0.0, 0.3, 30.0, 300.0):
+        pair = H.Pair(numels, 8, theta=0.0)
+        w, v = _params(numels, gen)
+        pair.attach(w, v)
+        pair.step(_make_rows(numels, 8, torch.float32, gen, k=k), "k=%g" % k)
+        pair.close()
+
+
+def test_large_offset_small_noise():
+    """Rows that agree to ~5 digits: the raw formula of App. B.3 would cancel, the shifted sums do not."""
+    gen = _gen(9)
+    n = 200000
+    base = torch.empty(n, device=DEV).normal_(100.0, 1.0, generator=gen)
+    rows = [[base + 1e-3 * torch.empty(n, device=DEV).normal_(0, 1, generator=gen)] for _ in range(8)]
+    pair = H.Pair([n], 8, theta=0.0)
+    w, v = _params([n], gen)
+    pair.attach(w, v)
+    pair.step(rows, "offset")
+    pair.close()
+
+
+def test_heavy_tailed_noise():
+    wl = synthetic.workload("transformer_base")
+    wl.shapes = [(50000,), (4096, 3), (17,)]
+    src = synthetic.GradientSource(wl, device=DEV)
+    wflat, vflat = src.init_params()
+    pair = H.Pair(src.numels, wl.S, momentum=0.99, lr=wl.lr)
+    pair.attach(src.views(wflat), src.views(vflat))
+    for step in range(3):
+        pair.step(src.fill(step), "student-t step %d" % step)
+    pair.close()
+
+
+@pytest.mark.parametrize("flags", [0, B.FLAG_LAGGED, B.FLAG_RATIO, B.FLAG_RATIO | B.FLAG_LAGGED, B.FLAG_CONT_TAU])
+@pytest.mark.parametrize("theta", [-1.0, 0.0, 0.7])
+def test_estimator_variants_and_theta(flags, theta):
+    gen = _gen(11)
+    numels = [5000, 129]
+    lr = {"kind": "exp", "eta0": 0.08, "d": 0.0133, "T_S1": 50.0}
+    pair = H.Pair(numels, 4, momentum=0.9, theta=theta, flags=flags, lr=lr)
+    w, v = _params(numels, gen)
+    pair.attach(w, v)
+    for step in range(6):
+        pair.step(_make_rows(numels, 4, torch.float32, gen, k=1.0 + step), "flags=%d step %d" % (flags, step),
+                  compare_tensors=(step % 3 == 0))
+    pair.close()
+
+
+def test_step_schedule_crosses_its_boundaries():
+    gen = _gen(12)
+    numels = [3000]
+    lr = {"kind": "step", "eta0": 0.1, "d": 0.1, "milestones": (5.0, 9.0, 14.0)}
+    pair = H.Pair(numels, 8, momentum=0.9, theta=0.0, lr=lr)
+    w, v = _params(numels, gen)
+    pair.attach(w, v)
+    seen = set()
+    for step in range(8):
+        st, _ = pair.step(_make_rows(numels, 8, torch.float32, gen, k=1.0), "sched step %d" % step)
+        seen.add(round(st.lr, 12))
+    assert len(seen) >= 3
+    pair.close()
+
+
+def test_elastic_scale_change():
+    gen = _gen(13)
+    numels = [2000, 31]
+    pair = H.Pair(numels, 4, momentum=0.9, max_S=16)
+    w, v = _params(numels, gen)
+    pair.attach(w, v)
+    for S in (4, 4, 8, 16, 16, 2):
+        pair.dev.set_scale(S)
+        pair.orc.set_scale(S)
+        pair.step(_make_rows(numels, S, torch.float32, gen), "elastic S=%d" % S)
+    with pytest.raises(B.AdaScaleError):
+        pair.dev.set_scale(17)
+    pair.close()
+
+
+def test_nonfinite_gradients_skip_the_step():
+    gen = _gen(14)
+    numels = [1000, 10]
+    pair = H.Pair(numels, 4, momentum=0.9)
+    w, v = _params(numels, gen)
+    pair.attach(w, v)
+    pair.step(_make_rows(numels, 4, torch.float32, gen), "before")
+    w0 = [t.clone() for t in w]
+    v0 = [t.clone() for t in v]
+    before = pair.dev.get_gain_tau(True)
+    rows = _make_rows(numels, 4, torch.float32, gen)
+    rows[2][0][17] = float("inf")
+    pair.dev.step(rows, w, v, pair.sched_dev)
+    st = pair.dev.get_gain_tau(True)
+    assert st.status_bits & B.STATUS_NONFINITE and st.skipped == 1 and st.eta == 0.0
+    assert st.tau == before.tau and st.t == before.t and st.sigma2_avg == before.sigma2_avg
+    for a, b in zip(w + v, w0 + v0):
+        assert torch.equal(a, b)
+    # the oracle applies the same policy, and the next clean step is in step with it again
+    rows_np = [[H.to_numpy_rows(g) for g in row] for row in rows]
+    ost = pair.orc.step(rows_np, pair.w64, pair.v64, pair.sched_orc)
+    assert ost["nonfinite"] == 1
+    pair.step(_make_rows(numels, 4, torch.float32, gen), "after")
+    assert pair.dev.get_gain_tau(True).status_bits == 0
+    pair.close()
+
+
+def test_bitwise_reproducible():
+    gen = _gen(15)
+    numels = [100000, 4097, 64]
+    rows = _make_rows(numels, 8, torch.float32, gen)
+    out = []
+    for _ in range(2):
+        g2 = _gen(16)
+        w, v = _params(numels, g2)
+        ada = B.AdaScale(numels, 8, momentum=0.9)
+        sched = B.make_schedule("const", eta0=0.1)
+        for _ in range(3):
+            ada.step(rows, w, v, sched)
+        st = ada.get_gain_tau(True)
+        out.append((st.as_dict(), [t.clone() for t in w + v]))
+        ada.close()
+    assert out[0][0] == out[1][0]
+    for a, b in zip(out[0][1], out[1][1]):
+        assert torch.equal(a, b)
+
+
+def test_checkpoint_resume_is_bitwise():
+    gen = _gen(17)
+    numels = [20000, 33]
+    steps = [_make_rows(numels, 4, torch.float32, gen, k=1.0 + i) for i in range(6)]
+    sched = B.make_schedule("exp", eta0=0.1, d=0.5, T_S1=10.0)
+
+    def run(split):
+        g2 = _gen(18)
+        w, v = _params(numels, g2)
+        ada = B.AdaScale(numels, 4, momentum=0.9, theta=0.6)
+        for i, rows in enumerate(steps):
+            if i == split:
+                blob = ada.get_state()
+                ada.close()
+                ada = B.AdaScale(numels, 4, momentum=0.9, theta=0.6)
+                ada.set_state(blob)
+            ada.step(rows, w, v, sched)
+        st = ada.get_gain_tau(True).as_dict()
+        ada.close()
+        return st, w, v
+
+    a, b = run(None), run(3)
+    assert a[0] == b[0]
+    for x, y in zip(a[1] + a[2], b[1] + b[2]):
+        assert torch.equal(x, y)
+    with pytest.raises(B.AdaScaleError):
+        ada = B.AdaScale(numels, 4)
+        ada.set_state(b"\0" * B.STATE_BYTES)
+
+
+def test_split_calls_equal_step_and_order_is_enforced():
+    gen = _gen(19)
+    numels = [5000]
+    rows = _make_rows(numels, 4, torch.float32, gen)
+    sched = B.make_schedule("const", eta0=0.1)
+    res = []
+    for split in (False, True):
+        w, v = _params(numels, _gen(20))
+        ada = B.AdaScale(numels, 4, momentum=0.9)
+        if split:
+            with pytest.raises(B.AdaScaleError) as e:
+                ada.update(w, v)
+            assert e.value.status == B.ERR_STATE
+            ada.reduce(rows, sched)
+            ada.update(w, v)
+        else:
+            ada.step(rows, w, v, sched)
+        torch.cuda.synchronize()
+        assert ada.launch_count == 2
+        res.append((w[0].clone(), v[0].clone()))
+        ada.close()
+    assert torch.equal(res[0][0], res[1][0]) and torch.equal(res[0][1], res[1][1])
+
+
+def test_host_gradients_entry_point():
+    gen = _gen(21)
+    numels = [3000, 64, 64, 100]
+    rows = _make_rows(numels, 4, torch.float32, gen)
+    sched = B.make_schedule("const", eta0=0.1)
+    w1, v1 = _params(numels, _gen(22))
+    w2, v2 = _params(numels, _gen(22))
+    a = B.AdaScale(numels, 4, momentum=0.9)
+    a.step(rows, w1, v1, sched)
+    s1 = a.get_gain_tau(True)
+    b = B.AdaScale(numels, 4, momentum=0.9)
+    host = [[g.cpu().pin_memory() for g in row] for row in rows]
+    s2 = b.step_host(host, w2, v2, sched)
+    assert s1.as_dict() == s2.as_dict()
+    for x, y in zip(w1 + v1, w2 + v2):
+        assert torch.equal(x, y)
+    a.close()
+    b.close()
+
+
+def test_error_paths_on_device():
+    numels = [16]
+    ada = B.AdaScale(numels, 2)
+    sched = B.make_schedule()
+    g = torch.zeros(64, device=DEV)
+    w = torch.zeros(16, device=DEV)
+    with pytest.raises(B.AdaScaleError) as e:
+        ada.step([0, g.data_ptr()], [w], [w.clone()], sched)
+    assert e.value.status == B.ERR_INVALID_ARG
+    with pytest.raises(B.AdaScaleError) as e:
+        ada.step([g.data_ptr() + 2, g.data_ptr()], [w], [w.clone()], sched)
+    assert e.value.status == B.ERR_ALIGNMENT
+    bad = B.make_schedule("exp", eta0=0.1, d=0.5, T_S1=0.0)
+    with pytest.raises(B.AdaScaleError):
+        ada.step([g, g], [w], [w.clone()], bad)
+    ada.close()
+
+
+def test_nonblocking_readback_trails_by_at_most_one_call():
+    gen = _gen(23)
+    numels = [1000]
+    ada = B.AdaScale(numels, 2)
+    w, v = _params(numels, gen)
+    sched = B.make_schedule()
+    rows = _make_rows(numels, 2, torch.float32, gen)
+    assert ada.get_gain_tau(False).t == 0
+    for _ in range(3):
+        ada.step(rows, w, v, sched)
+    ada.get_gain_tau(False)
+    torch.cuda.synchronize()
+    assert ada.get_gain_tau(False).t == 3
+    ada.close()

@@ -1,0 +1,115 @@
+"""The five benchmark workloads end to end against the oracle, at full size."""
+import math
+
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+if not torch.cuda.is_available():
+    pytest.skip("needs a CUDA device", allow_module_level=True)
+
+import _harness as H  # noqa: E402
+from paper_2007_05105_b200 import synthetic  # noqa: E402
+
+DEV = torch.device("cuda:0")
+
+
+def expected_gain(k, S):
+    return (k * k + 1.0) / (k * k / S + 1.0)
+
+
+def _pair(wl, src, **over):
+    pair = H.Pair(src.numels, wl.S, wl.grad_dtype, momentum=wl.momentum, weight_decay=wl.weight_decay,
+                  lr=wl.lr, **over)
+    w, v = src.init_params()
+    pair.attach(src.views(w), src.views(v))
+    return pair
+
+
+def test_single_tensor_1m_ten_steps():
+    wl = synthetic.workload("single_1m")
+    src = synthetic.GradientSource(wl, device=DEV)
+    pair = _pair(wl, src)
+    for step in range(wl.steps):
+        st, _ = pair.step(src.fill(step), "step %d" % step)
+    assert st.r == pytest.approx(expected_gain(10.0, 4), rel=0.02)  # 3.885
+    assert st.t == 10
+    pair.close()
+
+
+@pytest.mark.parametrize("k", [0.0, 0.3, 3.0, 30.0])
+def test_resnet18_noise_sweep(k):
+    wl = synthetic.workload("resnet18", k=(k, k))
+    src = synthetic.GradientSource(wl, device=DEV)
+    pair = _pair(wl, src)
+    steps = 10 if k == 3.0 else 3  # k = 3: tau passes the boundaries at 20 and 40
+    lrs = set()
+    for step in range(steps):
+        st, _ = pair.step(src.fill(step), "k=%g step %d" % (k, step), compare_tensors=(step in (0, steps - 1)))
+        lrs.add(round(st.lr, 12))
+    assert st.r == pytest.approx(expected_gain(k, 8), rel=0.02)
+    if k == 3.0:
+        assert lrs == {0.1, 0.01, 0.001}
+    pair.close()
+
+
+def test_resnet50_bf16_full_size_steps():
+    wl = synthetic.workload("resnet50")
+    src = synthetic.GradientSource(wl, device=DEV)
+    pair = _pair(wl, src)
+    for step in range(4):
+        st, _ = pair.step(src.fill(step), "step %d" % step, compare_tensors=(step in (0, 3)))
+    assert st.r == pytest.approx(expected_gain(3.0, 16), rel=0.03)  # 6.40
+    pair.close()
+
+
+def test_resnet50_bf16_thousand_step_clock():
+    """tau after 1000 iterations against the oracle (reduced width so the oracle keeps up)."""
+    wl = synthetic.workload("resnet50")
+    wl.shapes = synthetic.resnet50_shapes(width=16, classes=100)
+    src = synthetic.GradientSource(wl, device=DEV)
+    pair = _pair(wl, src)
+    total = 0.0
+    for step in range(1000):
+        st, ost = pair.step(src.fill(step), "step %d" % step, compare_tensors=(step % 250 == 0))
+        total += st.r
+    assert abs(st.tau - ost["tau"]) <= 1e-4 * ost["tau"]
+    assert st.tau == pytest.approx(total, rel=1e-12)
+    assert st.t == 1000 and math.ceil(st.tau / 16) <= 1000 <= st.tau
+    pair.close()
+
+
+def test_transformer_base_heavy_tails_full_size():
+    wl = synthetic.workload("transformer_base")
+    src = synthetic.GradientSource(wl, device=DEV)
+    pair = _pair(wl, src)
+    sample = [0, 1, 2, 9, 100, 256]
+    for step in range(2):
+        st, _ = pair.step_streamed(src.fill(step), "step %d" % step, sample_tensors=sample)
+    assert 1.0 <= st.r <= 32.0
+    pair.close()
+
+
+def test_decoder_24l_bf16_full_size():
+    wl = synthetic.workload("decoder_24l")
+    src = synthetic.GradientSource(wl, device=DEV)
+    pair = _pair(wl, src)
+    sample = [0, 1, 2, 3, 150, 291]
+    for step, k in enumerate((0.1, 10.0)):
+        st, _ = pair.step_streamed(src.fill(step, k=k), "k=%g" % k, sample_tensors=sample)
+    pair.close()
+
+
+def test_decoder_drifting_noise_200_steps_reduced():
+    """k drifts 0.1 -> 10 over 200 steps; the gain follows behind the moving average."""
+    wl = synthetic.workload("decoder_24l")
+    wl.shapes = synthetic.decoder_24l_shapes(d=128, ffn=512, layers=2, vocab=1000, positions=64)
+    src = synthetic.GradientSource(wl, device=DEV)
+    pair = _pair(wl, src)
+    rs = []
+    for step in range(200):
+        st, _ = pair.step(src.fill(step), "step %d" % step, compare_tensors=(step % 50 == 0))
+        rs.append(st.r)
+    assert rs[0] < 1.1 and rs[-1] > 10.0
+    pair.close()
