@@ -137,61 +137,95 @@ template <> struct Elem<ADASCALE_BF16> {
 // ---------------------------------------------------------------------------------------
 // One column vector (4 fp32 or 8 bf16 columns) of all S rows.
 //
-// Per column the S values are shifted by the first row's value c:  d_i = g_i - c.  With
-// s1 = sum d_i and s2 = sum d_i^2 the mean is c + s1/S and the summed squared deviation is
-// s2 - s1^2/S.  The shift is itself a sample, so the subtraction loses a factor of order S
-// at worst (not the |mean|^2/sigma^2 of the raw formula of App. B.3), identical rows give
-// exactly zero, and each row is consumed as it arrives: no register array of S rows.
+// Per column the S values are shifted by a value c taken from the data:  d_i = g_i - c.
+// With s1 = sum d_i and s2 = sum d_i^2 the mean is c + s1/S and the summed squared
+// deviation is s2 - s1^2/S.  Because c is itself (close to) a sample, the subtraction
+// loses a factor of order S at worst, not the |mean|^2/sigma^2 that the raw formula of
+// App. B.3 loses; identical rows give exactly zero; and every row is consumed as it
+// arrives, so no register array of S rows is needed.
+//   - c is the median of the first three rows (row 0 when fewer than four rows are
+//     fetched together): one outlier among them cannot become the shift, which keeps
+//     |s1| and with it the rounding error of the mean small under heavy-tailed noise.
+//   - s1 is summed in blocks of B rows (a fresh partial per block, then one add), so the
+//     long chain of roundings happens on small partial sums.
 // B <= S rows are requested together to keep 16*B bytes per thread in flight.
 // ---------------------------------------------------------------------------------------
+template <int V>
+__device__ __forceinline__ void accumulate_row(const float *x, const float *c, float *p1, float *s2)
+{
+#pragma unroll
+    for (int k = 0; k < V; ++k) {
+        const float d = x[k] - c[k];
+        p1[k] += d;
+        s2[k] = fmaf(d, d, s2[k]);
+    }
+}
+
 template <int DT, int B>
 __device__ __forceinline__ void column_vector(const u64 *rowp, size_t boff, int S, float invS, float fS,
                                               float *gb, float &dsum, float &nsum)
 {
     constexpr int V = Elem<DT>::kVec;
-    float c[V], s1[V], s2[V], x[V];
+    float c[V], s1[V], s2[V], p1[V], x[V];
 #pragma unroll
-    for (int k = 0; k < V; ++k) s1[k] = s2[k] = 0.f;
+    for (int k = 0; k < V; ++k) s1[k] = s2[k] = p1[k] = 0.f;
 
     uint4 q[B];
-    // first batch: rows 0 .. B-1 (row 0 is the shift)
 #pragma unroll
     for (int b = 0; b < B; ++b) q[b] = ld_stream16((const char *)rowp[b] + boff);
-    Elem<DT>::unpack(q[0], c);
-#pragma unroll
-    for (int b = 1; b < B; ++b) {
-        Elem<DT>::unpack(q[b], x);
+    if (B >= 4) {
+        float x1[V], x2[V];
+        Elem<DT>::unpack(q[0], x);
+        Elem<DT>::unpack(q[1], x1);
+        Elem<DT>::unpack(q[2], x2);
 #pragma unroll
         for (int k = 0; k < V; ++k) {
-            float d = x[k] - c[k];
-            s1[k] += d;
-            s2[k] = fmaf(d, d, s2[k]);
+            const float lo = fminf(x[k], x1[k]), hi = fmaxf(x[k], x1[k]);
+            c[k] = fmaxf(lo, fminf(hi, x2[k]));  // median of three
+        }
+        accumulate_row<V>(x, c, p1, s2);
+        accumulate_row<V>(x1, c, p1, s2);
+        accumulate_row<V>(x2, c, p1, s2);
+#pragma unroll
+        for (int b = 3; b < B; ++b) {
+            Elem<DT>::unpack(q[b], x);
+            accumulate_row<V>(x, c, p1, s2);
+        }
+    } else {
+        Elem<DT>::unpack(q[0], c);  // d_0 = 0
+#pragma unroll
+        for (int b = 1; b < B; ++b) {
+            Elem<DT>::unpack(q[b], x);
+            accumulate_row<V>(x, c, p1, s2);
         }
     }
+#pragma unroll
+    for (int k = 0; k < V; ++k) s1[k] = p1[k];
+
     int i = B;
     for (; i + B <= S; i += B) {
 #pragma unroll
         for (int b = 0; b < B; ++b) q[b] = ld_stream16((const char *)rowp[i + b] + boff);
 #pragma unroll
+        for (int k = 0; k < V; ++k) p1[k] = 0.f;
+#pragma unroll
         for (int b = 0; b < B; ++b) {
             Elem<DT>::unpack(q[b], x);
-#pragma unroll
-            for (int k = 0; k < V; ++k) {
-                float d = x[k] - c[k];
-                s1[k] += d;
-                s2[k] = fmaf(d, d, s2[k]);
-            }
+            accumulate_row<V>(x, c, p1, s2);
         }
+#pragma unroll
+        for (int k = 0; k < V; ++k) s1[k] += p1[k];
     }
-    for (; i < S; ++i) {
-        q[0] = ld_stream16((const char *)rowp[i] + boff);
-        Elem<DT>::unpack(q[0], x);
+    if (i < S) {
 #pragma unroll
-        for (int k = 0; k < V; ++k) {
-            float d = x[k] - c[k];
-            s1[k] += d;
-            s2[k] = fmaf(d, d, s2[k]);
+        for (int k = 0; k < V; ++k) p1[k] = 0.f;
+        for (; i < S; ++i) {
+            q[0] = ld_stream16((const char *)rowp[i] + boff);
+            Elem<DT>::unpack(q[0], x);
+            accumulate_row<V>(x, c, p1, s2);
         }
+#pragma unroll
+        for (int k = 0; k < V; ++k) s1[k] += p1[k];
     }
 
     float m[V];
@@ -201,7 +235,7 @@ __device__ __forceinline__ void column_vector(const u64 *rowp, size_t boff, int 
         // quotient s1/S: reciprocal multiply plus one residual correction (1/S is not exact
         // unless S is a power of two, and a biased 1/S would bias every column the same way)
         float qk = s1[k] * invS;
-        float res = fmaf(-qk, fS, s1[k]);
+        const float res = fmaf(-qk, fS, s1[k]);
         qk = fmaf(res, invS, qk);
         m[k] = c[k] + qk;
         dacc += fmaf(-qk, s1[k], s2[k]);
