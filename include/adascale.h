@@ -91,7 +91,9 @@ typedef struct {
 } adascale_config;
 
 /* status bits reported in adascale_stats.status_bits */
-#define ADASCALE_STATUS_NONFINITE 1u /* last step saw inf/nan sums and was skipped */
+#define ADASCALE_STATUS_NONFINITE 1u    /* last step saw inf/nan sums and was skipped           */
+#define ADASCALE_STATUS_WAIT_TIMEOUT 2u /* sticky: a bounded wait inside a kernel gave up; the
+                                           results of that step and later ones are not valid    */
 
 typedef struct {
     double r;           /* gain ratio r_t of the last step                            */
@@ -209,6 +211,17 @@ adascale_status adascale_step_host(adascale_ctx *ctx, const void *const *grads, 
  * multiple of 16.  One launch on `cuda_stream`.
  */
 adascale_status adascale_stream_probe(int32_t kind, void *a, void *b, int64_t n_bytes, void *cuda_stream);
+
+/*
+ * Host-only view of how the library splits a tensor list over the blocks of its persistent
+ * kernels (no counterpart in the paper; used by tests).  numel: host array [n_tensors];
+ * unit: elements per vector access; seg_cost: fixed cost of a segment in units;
+ * max_blocks: grid size.  Writes up to cap rows of 4 int64 {tensor, first element, length
+ * in elements, block} into out, in block order, and returns the number of segments
+ * (which may exceed cap), or -1 for invalid arguments.  Makes no CUDA call.
+ */
+int64_t adascale_plan(const int64_t *numel, int32_t n_tensors, int32_t unit, int64_t seg_cost,
+                      int32_t max_blocks, int64_t *out, int64_t cap);
 
 /* Number of kernels the library has launched through this context since init. */
 int64_t adascale_launch_count(const adascale_ctx *ctx);

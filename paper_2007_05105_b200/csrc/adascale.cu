@@ -14,6 +14,7 @@
 
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -23,19 +24,29 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
-constexpr int kChunkF32 = 2048;   // elements one block handles (fp32 gradients)
-constexpr int kChunkBF16 = 4096;  // elements one block handles (bf16 gradients)
+constexpr int kReduceBlocksPerSM = 4;  // resident blocks the reduce kernel is compiled for
+constexpr int kUpdateBlocksPerSM = 8;  // same for the update kernel
+constexpr int kMinUnitsPerBlock = 512; // do not spread a small job over more blocks than this allows
 constexpr int kGbarAlign = 64;    // every tensor's mean gradient starts on a 256-byte boundary
 constexpr int kRing = 4;          // pinned staging slots for pointer-table uploads
 constexpr int kMaxS = 4096;
 
 typedef unsigned long long u64;
 
-struct Chunk {
+// A contiguous run of elements of one tensor, owned by one block.
+struct Segment {
     long long off;   // first element inside the tensor
     long long goff;  // first element inside the mean-gradient workspace
     int tensor;
-    int len;
+    int len;         // elements
+};
+
+// Static split of all tensors over the blocks of a persistent grid: block b owns
+// segs[first[b]] .. segs[first[b+1]-1].  Built once on the host (see make_plan).
+struct Plan {
+    std::vector<Segment> segs;
+    std::vector<int> first;  // n_blocks + 1 entries
+    int n_blocks = 0;
 };
 
 // Scalar state kept on the device between iterations.
@@ -50,7 +61,7 @@ struct DevState {
     double sigma2_raw, mu2_raw;
     double N, D;
     unsigned status;
-    unsigned pad;
+    unsigned fault;  // sticky: a bounded device-side wait gave up
 };
 
 struct ScalarCfg {
@@ -66,26 +77,28 @@ struct Sched {
 };
 
 struct ReduceArgs {
-    const Chunk *chunks;
+    const Segment *segs;
+    const int *first;
     const u64 *gptr;        // [S * T] row pointers
     const unsigned *gflags; // [T] bit0: all S rows of the tensor are 16-byte aligned
     float *gbar;
     double2 *partials;
     unsigned *ticket;
     DevState *st;
-    int n_chunks, S, T;
+    int S, T;
     float invS, fS;
     ScalarCfg sc;
     Sched sched;
 };
 
 struct UpdateArgs {
-    const Chunk *chunks;
+    const Segment *segs;
+    const int *first;
     const u64 *wv;          // [2 * T]: parameters then momentum
     const unsigned *wflags; // [T] bit0: both pointers 16-byte aligned
     const float *gbar;
     const DevState *st;
-    int n_chunks, T;
+    int T;
     float rho, lambda;
 };
 
@@ -268,6 +281,27 @@ __device__ __forceinline__ void column_scalar(const u64 *rowp, size_t boff, int 
     nsum = m * m;
 }
 
+// Same, with the row pointers read from the device table instead of shared memory.
+template <int DT>
+__device__ __forceinline__ void column_scalar_direct(const u64 *gptr, int T, int tensor, size_t boff, int S,
+                                                     float fS, float *gb, float &dsum, float &nsum)
+{
+    float sum = 0.f;
+    for (int i = 0; i < S; ++i) sum += Elem<DT>::load1((const char *)gptr[(size_t)i * T + tensor] + boff);
+    const float m0 = sum / fS;
+    float e = 0.f, qq = 0.f;
+    for (int i = 0; i < S; ++i) {
+        const float d = Elem<DT>::load1((const char *)gptr[(size_t)i * T + tensor] + boff) - m0;
+        e += d;
+        qq = fmaf(d, d, qq);
+    }
+    const float corr = e / fS;
+    const float m = m0 + corr;
+    *gb = m;
+    dsum = fmaf(-corr, e, qq);
+    nsum = m * m;
+}
+
 __device__ __forceinline__ double warp_sum(double v)
 {
 #pragma unroll
@@ -275,7 +309,8 @@ __device__ __forceinline__ double warp_sum(double v)
     return v;
 }
 
-// Fixed-shape block sum of two doubles; result valid in thread 0.
+// Fixed-shape block sum of two doubles over NW warps; result valid in thread 0.
+template <int NW = kWarps>
 __device__ __forceinline__ void block_sum2(double &a, double &b, double *sa, double *sb)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -288,8 +323,8 @@ __device__ __forceinline__ void block_sum2(double &a, double &b, double *sa, dou
     }
     __syncthreads();
     if (warp == 0) {
-        a = lane < kWarps ? sa[lane] : 0.0;
-        b = lane < kWarps ? sb[lane] : 0.0;
+        a = lane < NW ? sa[lane] : 0.0;
+        b = lane < NW ? sb[lane] : 0.0;
         a = warp_sum(a);
         b = warp_sum(b);
     }
@@ -374,8 +409,10 @@ __device__ void scalar_step(DevState *st, const ScalarCfg &c, const Sched &sched
     st->t += 1;
 }
 
+// Persistent grid: every block walks its own segments and keeps two fp64 accumulators per
+// thread for the whole launch, so there is one block reduction and one partial pair per block.
 template <int DT, int B>
-__global__ void __launch_bounds__(kThreads) k_reduce(const __grid_constant__ ReduceArgs a)
+__global__ void __launch_bounds__(kThreads, kReduceBlocksPerSM) k_reduce(const __grid_constant__ ReduceArgs a)
 {
     extern __shared__ u64 rowp[];
     __shared__ double sa[kWarps], sb[kWarps];
@@ -384,29 +421,34 @@ __global__ void __launch_bounds__(kThreads) k_reduce(const __grid_constant__ Red
     constexpr int V = Elem<DT>::kVec;
     constexpr int E = Elem<DT>::kBytes;
     const int tid = threadIdx.x;
-    const Chunk ch = a.chunks[blockIdx.x];
-    for (int i = tid; i < a.S; i += kThreads)
-        rowp[i] = a.gptr[(size_t)i * a.T + ch.tensor] + (u64)ch.off * E;
-    __syncthreads();
-
-    float *gb = a.gbar + ch.goff;
     double accD = 0.0, accN = 0.0;
-    int first_scalar = 0;
-    if (a.gflags[ch.tensor] & 1u) {
-        const int nv = ch.len / V;
-        for (int v = tid; v < nv; v += kThreads) {
+
+    const int seg_end = a.first[blockIdx.x + 1];
+    for (int sidx = a.first[blockIdx.x]; sidx < seg_end; ++sidx) {
+        const Segment sg = a.segs[sidx];
+        __syncthreads();  // the previous segment's row pointers are no longer needed
+        for (int i = tid; i < a.S; i += kThreads)
+            rowp[i] = a.gptr[(size_t)i * a.T + sg.tensor] + (u64)sg.off * E;
+        __syncthreads();
+
+        float *gb = a.gbar + sg.goff;
+        int first_scalar = 0;
+        if (a.gflags[sg.tensor] & 1u) {
+            const int nv = sg.len / V;
+            for (int v = tid; v < nv; v += kThreads) {
+                float d, n;
+                column_vector<DT, B>(rowp, (size_t)v * 16, a.S, a.invS, a.fS, gb + (size_t)v * V, d, n);
+                accD += (double)d;
+                accN += (double)n;
+            }
+            first_scalar = nv * V;
+        }
+        for (int e = first_scalar + tid; e < sg.len; e += kThreads) {
             float d, n;
-            column_vector<DT, B>(rowp, (size_t)v * 16, a.S, a.invS, a.fS, gb + (size_t)v * V, d, n);
+            column_scalar<DT>(rowp, (size_t)e * E, a.S, a.fS, gb + e, d, n);
             accD += (double)d;
             accN += (double)n;
         }
-        first_scalar = nv * V;
-    }
-    for (int e = first_scalar + tid; e < ch.len; e += kThreads) {
-        float d, n;
-        column_scalar<DT>(rowp, (size_t)e * E, a.S, a.fS, gb + e, d, n);
-        accD += (double)d;
-        accN += (double)n;
     }
 
     block_sum2(accD, accN, sa, sb);
@@ -420,7 +462,7 @@ __global__ void __launch_bounds__(kThreads) k_reduce(const __grid_constant__ Red
     if (!is_last) return;
 
     // Second stage, fixed order: thread j adds partials j, j+256, ... in index order, then the
-    // same block tree.  The result depends on the chunk table only, not on block scheduling.
+    // same block tree.  The result depends on the plan only, not on how blocks were scheduled.
     __threadfence();
     double d = 0.0, n = 0.0;
     for (int i = tid; i < (int)gridDim.x; i += kThreads) {
@@ -435,40 +477,329 @@ __global__ void __launch_bounds__(kThreads) k_reduce(const __grid_constant__ Red
     }
 }
 
-__global__ void __launch_bounds__(kThreads) k_update(const __grid_constant__ UpdateArgs a)
+// ---------------------------------------------------------------------------------------
+// Reduce kernel, staged variant: a producer warp streams tiles of the gradient matrix into
+// shared memory with bulk asynchronous copies (one copy per row per tile, completion counted
+// on an mbarrier), eight consumer warps read the tiles back from shared memory.  Memory
+// latency is covered by the stages in flight instead of by registers, and the consumers
+// issue no global loads or address arithmetic at all.
+//
+// A work item is (segment, column tile, row chunk): kTileThreads * CPT columns of up to
+// kRowsPerStage rows.  Row chunks let any S through: the per-column sums carry over from one
+// chunk of rows to the next and are closed after the last.
+// ---------------------------------------------------------------------------------------
+constexpr int kStages = 3;
+constexpr int kRowsPerStage = 32;
+constexpr int kConsumers = kThreads;          // 8 consumer warps
+constexpr int kStagedThreads = kThreads + 32; // + 1 producer warp
+constexpr int kStagedWarps = kStagedThreads / 32;
+constexpr unsigned kSpinLimit = 1u << 22;     // bounded waits: give up, flag, leave
+
+__device__ __forceinline__ unsigned smem_u32(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(u64 *bar, unsigned count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(u64 *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(u64 *bar, unsigned bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Returns false if the phase did not complete within the spin limit.
+__device__ __forceinline__ bool mbar_wait(u64 *bar, unsigned parity)
+{
+    const unsigned addr = smem_u32(bar);
+    for (unsigned spin = 0; spin < kSpinLimit; ++spin) {
+        unsigned done;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done)
+                     : "r"(addr), "r"(parity)
+                     : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+// global -> shared bulk copy; bytes and both addresses are multiples of 16.  The rows are read
+// once: evict-first in L2 leaves the cache to the mean gradient that the update reads next.
+__device__ __forceinline__ void bulk_load(void *dst, const void *src, unsigned bytes, u64 *bar, u64 policy)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
+                 : "memory");
+}
+
+template <int DT, int CPT> struct Cols;
+template <int CPT> struct Cols<ADASCALE_F32, CPT> {
+    static __device__ __forceinline__ void load(const char *p, float *x)
+    {
+        if constexpr (CPT == 1) {
+            x[0] = *(const float *)p;
+        } else if constexpr (CPT == 2) {
+            const float2 t = *(const float2 *)p;
+            x[0] = t.x; x[1] = t.y;
+        } else {
+#pragma unroll
+            for (int k = 0; k < CPT; k += 4) {
+                const float4 t = *(const float4 *)(p + 4 * k);
+                x[k] = t.x; x[k + 1] = t.y; x[k + 2] = t.z; x[k + 3] = t.w;
+            }
+        }
+    }
+};
+template <int CPT> struct Cols<ADASCALE_BF16, CPT> {
+    static __device__ __forceinline__ void widen(unsigned u, float *x)
+    {
+        x[0] = __uint_as_float(u << 16);
+        x[1] = __uint_as_float(u & 0xffff0000u);
+    }
+    static __device__ __forceinline__ void load(const char *p, float *x)
+    {
+        if constexpr (CPT == 2) {
+            widen(*(const unsigned *)p, x);
+        } else if constexpr (CPT == 4) {
+            const uint2 t = *(const uint2 *)p;
+            widen(t.x, x); widen(t.y, x + 2);
+        } else {
+            const uint4 t = *(const uint4 *)p;
+            widen(t.x, x); widen(t.y, x + 2); widen(t.z, x + 4); widen(t.w, x + 6);
+        }
+    }
+};
+
+template <int CPT>
+__device__ __forceinline__ void store_cols(float *g, const float *m)
+{
+    if constexpr (CPT == 1) {
+        g[0] = m[0];
+    } else if constexpr (CPT == 2) {
+        *(float2 *)g = make_float2(m[0], m[1]);
+    } else {
+#pragma unroll
+        for (int k = 0; k < CPT; k += 4) *(float4 *)(g + k) = make_float4(m[k], m[k + 1], m[k + 2], m[k + 3]);
+    }
+}
+
+template <int DT, int CPT>
+__global__ void __launch_bounds__(kStagedThreads, 2) k_reduce_staged(const __grid_constant__ ReduceArgs a)
+{
+    extern __shared__ __align__(128) unsigned char stage_mem[];
+    __shared__ __align__(8) u64 full_bar[kStages], empty_bar[kStages];
+    __shared__ double sa[kStagedWarps], sb[kStagedWarps];
+    __shared__ bool is_last;
+    __shared__ int abort_flag;
+
+    constexpr int E = Elem<DT>::kBytes;
+    constexpr int kTile = kConsumers * CPT;     // columns per tile
+    constexpr int kRowBytes = kTile * E;        // one row of a stage
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const bool producer = warp == kStagedWarps - 1;
+    const int S = a.S;
+    const int rps = S < kRowsPerStage ? S : kRowsPerStage;  // rows per stage
+    const int n_chunks = (S + rps - 1) / rps;
+    const unsigned stage_bytes = (unsigned)rps * kRowBytes;
+
+    if (tid == 0) {
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(&full_bar[i], 1);
+            mbar_init(&empty_bar[i], kConsumers / 32);
+        }
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    double accD = 0.0, accN = 0.0;
+    unsigned item = 0;  // running count of staged work items, identical in every thread
+    bool timed_out = false;
+    const int seg_end = a.first[blockIdx.x + 1];
+
+    if (producer) {
+        u64 policy;
+        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+        int last_use[kStages];
+#pragma unroll
+        for (int i = 0; i < kStages; ++i) last_use[i] = -1;
+        for (int sidx = a.first[blockIdx.x]; sidx < seg_end && !timed_out; ++sidx) {
+            const Segment sg = a.segs[sidx];
+            if (!(a.gflags[sg.tensor] & 1u)) continue;  // consumers take unaligned tensors from global memory
+            const int cols = sg.len & ~7;
+            for (int c0 = 0; c0 < cols && !timed_out; c0 += kTile) {
+                const int tc = cols - c0 < kTile ? cols - c0 : kTile;
+                for (int ch = 0; ch < n_chunks; ++ch, ++item) {
+                    const int st = item % kStages;
+                    const unsigned use = item / kStages;
+                    if (!mbar_wait(&empty_bar[st], (use & 1u) ^ 1u)) { timed_out = true; break; }
+                    const int r0 = ch * rps;
+                    const int rows = S - r0 < rps ? S - r0 : rps;
+                    if (lane == 0) mbar_expect_tx(&full_bar[st], (unsigned)rows * tc * E);
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < kStages; ++i)
+                        if (i == st) last_use[i] = (int)use;
+                    for (int r = lane; r < rows; r += 32) {
+                        const char *src = (const char *)a.gptr[(size_t)(r0 + r) * a.T + sg.tensor] + ((size_t)sg.off + c0) * E;
+                        bulk_load(stage_mem + (size_t)st * stage_bytes + (size_t)r * kRowBytes, src, (unsigned)tc * E,
+                                  &full_bar[st], policy);
+                    }
+                }
+            }
+        }
+        if (timed_out) atomicExch(&abort_flag, 1);
+        if (timed_out || *(volatile int *)&abort_flag) {
+            // leaving early: copies already issued must land before this block's shared memory is reused
+#pragma unroll
+            for (int i = 0; i < kStages; ++i)
+                if (last_use[i] >= 0) mbar_wait(&full_bar[i], (unsigned)last_use[i] & 1u);
+        }
+    } else {
+        float c[CPT], s1[CPT], s2[CPT], p1[CPT], x[CPT];
+        for (int sidx = a.first[blockIdx.x]; sidx < seg_end && !timed_out; ++sidx) {
+            const Segment sg = a.segs[sidx];
+            float *gb = a.gbar + sg.goff;
+            int first_scalar = 0;
+            if (a.gflags[sg.tensor] & 1u) {
+                const int cols = sg.len & ~7;
+                first_scalar = cols;
+                for (int c0 = 0; c0 < cols && !timed_out; c0 += kTile) {
+                    const int tc = cols - c0 < kTile ? cols - c0 : kTile;
+                    const bool active = tid * CPT < tc;
+                    for (int ch = 0; ch < n_chunks; ++ch, ++item) {
+                        const int st = item % kStages;
+                        const unsigned use = item / kStages;
+                        if (!mbar_wait(&full_bar[st], use & 1u)) { timed_out = true; break; }
+                        const int r0 = ch * rps;
+                        const int rows = S - r0 < rps ? S - r0 : rps;
+                        const char *base = (const char *)stage_mem + (size_t)st * stage_bytes + (size_t)tid * CPT * E;
+                        if (active) {
+                            if (ch == 0) {
+                                if (S >= 3) {  // shift = median of the first three rows
+                                    float x1[CPT], x2[CPT];
+                                    Cols<DT, CPT>::load(base, x);
+                                    Cols<DT, CPT>::load(base + kRowBytes, x1);
+                                    Cols<DT, CPT>::load(base + 2 * kRowBytes, x2);
+#pragma unroll
+                                    for (int k = 0; k < CPT; ++k) {
+                                        const float lo = fminf(x[k], x1[k]), hi = fmaxf(x[k], x1[k]);
+                                        c[k] = fmaxf(lo, fminf(hi, x2[k]));
+                                    }
+                                } else {
+                                    Cols<DT, CPT>::load(base, c);
+                                }
+#pragma unroll
+                                for (int k = 0; k < CPT; ++k) s1[k] = s2[k] = 0.f;
+                            }
+                            for (int r = 0; r < rows; r += 8) {  // s1 in blocks of 8 rows
+#pragma unroll
+                                for (int k = 0; k < CPT; ++k) p1[k] = 0.f;
+#pragma unroll
+                                for (int rr = 0; rr < 8; ++rr) {
+                                    if (r + rr < rows) {
+                                        Cols<DT, CPT>::load(base + (size_t)(r + rr) * kRowBytes, x);
+                                        accumulate_row<CPT>(x, c, p1, s2);
+                                    }
+                                }
+#pragma unroll
+                                for (int k = 0; k < CPT; ++k) s1[k] += p1[k];
+                            }
+                        }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&empty_bar[st]);  // this warp is done with the stage
+                        if (active && ch == n_chunks - 1) {
+                            float m[CPT];
+                            float dacc = 0.f, nacc = 0.f;
+#pragma unroll
+                            for (int k = 0; k < CPT; ++k) {
+                                float qk = s1[k] * a.invS;
+                                const float res = fmaf(-qk, a.fS, s1[k]);
+                                qk = fmaf(res, a.invS, qk);
+                                m[k] = c[k] + qk;
+                                dacc += fmaf(-qk, s1[k], s2[k]);
+                                nacc = fmaf(m[k], m[k], nacc);
+                            }
+                            store_cols<CPT>(gb + c0 + tid * CPT, m);
+                            accD += (double)dacc;
+                            accN += (double)nacc;
+                        }
+                    }
+                }
+            }
+            // ragged tail (< 8 elements) or a tensor that is not 16-byte aligned: plain loads
+            for (int e = first_scalar + tid; e < sg.len && !timed_out; e += kConsumers) {
+                float d, n;
+                column_scalar_direct<DT>(a.gptr, a.T, sg.tensor, ((size_t)sg.off + e) * E, S, a.fS, gb + e, d, n);
+                accD += (double)d;
+                accN += (double)n;
+            }
+        }
+        if (timed_out) atomicExch(&abort_flag, 1);
+    }
+
+    block_sum2<kStagedWarps>(accD, accN, sa, sb);
+    if (tid == 0) {
+        if (abort_flag) atomicOr(&a.st->fault, ADASCALE_STATUS_WAIT_TIMEOUT);
+        a.partials[blockIdx.x] = make_double2(accD, accN);
+        __threadfence();
+        const unsigned tk = atomicAdd(a.ticket, 1u);
+        is_last = (tk == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+
+    __threadfence();
+    double d = 0.0, n = 0.0;
+    for (int i = tid; i < (int)gridDim.x; i += kStagedThreads) {
+        const double2 p = __ldcg(&a.partials[i]);
+        d += p.x;
+        n += p.y;
+    }
+    block_sum2<kStagedWarps>(d, n, sa, sb);
+    if (tid == 0) {
+        scalar_step(a.st, a.sc, a.sched, d, n);
+        *a.ticket = 0u;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const __grid_constant__ UpdateArgs a)
 {
     if (a.st->status & ADASCALE_STATUS_NONFINITE) return;
     const float eta = (float)a.st->eta;
-    // newest mean-gradient chunks first: they are the most likely to still sit in L2
-    const Chunk ch = a.chunks[a.n_chunks - 1 - (int)blockIdx.x];
-    float *w = (float *)a.wv[ch.tensor] + ch.off;
-    float *v = (float *)a.wv[a.T + ch.tensor] + ch.off;
-    const float *g = a.gbar + ch.goff;
     const int tid = threadIdx.x;
-    int first_scalar = 0;
-    if (a.wflags[ch.tensor] & 1u) {
-        const int nv = ch.len >> 2;
-        for (int i = tid; i < nv; i += kThreads) {
-            const float4 gg = ((const float4 *)g)[i];
-            float4 ww = ((const float4 *)w)[i];
-            float4 vv = ((const float4 *)v)[i];
-            vv.x = fmaf(a.rho, vv.x, fmaf(a.lambda, ww.x, gg.x));
-            vv.y = fmaf(a.rho, vv.y, fmaf(a.lambda, ww.y, gg.y));
-            vv.z = fmaf(a.rho, vv.z, fmaf(a.lambda, ww.z, gg.z));
-            vv.w = fmaf(a.rho, vv.w, fmaf(a.lambda, ww.w, gg.w));
-            ww.x = fmaf(-eta, vv.x, ww.x);
-            ww.y = fmaf(-eta, vv.y, ww.y);
-            ww.z = fmaf(-eta, vv.z, ww.z);
-            ww.w = fmaf(-eta, vv.w, ww.w);
-            ((float4 *)v)[i] = vv;
-            ((float4 *)w)[i] = ww;
+    const int seg_end = a.first[blockIdx.x + 1];
+    for (int sidx = a.first[blockIdx.x]; sidx < seg_end; ++sidx) {
+        const Segment sg = a.segs[sidx];
+        float *w = (float *)a.wv[sg.tensor] + sg.off;
+        float *v = (float *)a.wv[a.T + sg.tensor] + sg.off;
+        const float *g = a.gbar + sg.goff;
+        int first_scalar = 0;
+        if (a.wflags[sg.tensor] & 1u) {
+            const int nv = sg.len >> 2;
+            for (int i = tid; i < nv; i += kThreads) {
+                const float4 gg = ((const float4 *)g)[i];
+                float4 ww = ((const float4 *)w)[i];
+                float4 vv = ((const float4 *)v)[i];
+                vv.x = fmaf(a.rho, vv.x, fmaf(a.lambda, ww.x, gg.x));
+                vv.y = fmaf(a.rho, vv.y, fmaf(a.lambda, ww.y, gg.y));
+                vv.z = fmaf(a.rho, vv.z, fmaf(a.lambda, ww.z, gg.z));
+                vv.w = fmaf(a.rho, vv.w, fmaf(a.lambda, ww.w, gg.w));
+                ww.x = fmaf(-eta, vv.x, ww.x);
+                ww.y = fmaf(-eta, vv.y, ww.y);
+                ww.z = fmaf(-eta, vv.z, ww.z);
+                ww.w = fmaf(-eta, vv.w, ww.w);
+                ((float4 *)v)[i] = vv;
+                ((float4 *)w)[i] = ww;
+            }
+            first_scalar = nv << 2;
         }
-        first_scalar = nv << 2;
-    }
-    for (int e = first_scalar + tid; e < ch.len; e += kThreads) {
-        const float vn = fmaf(a.rho, v[e], fmaf(a.lambda, w[e], g[e]));
-        v[e] = vn;
-        w[e] = fmaf(-eta, vn, w[e]);
+        for (int e = first_scalar + tid; e < sg.len; e += kThreads) {
+            const float vn = fmaf(a.rho, v[e], fmaf(a.lambda, w[e], g[e]));
+            v[e] = vn;
+            w[e] = fmaf(-eta, vn, w[e]);
+        }
     }
 }
 
@@ -540,8 +871,10 @@ struct adascale_ctx {
     std::vector<long long> numel;
     std::vector<long long> goff;
     long long P = 0, gbar_elems = 0;
-    int n_chunks = 0;
-    Chunk *d_chunks = nullptr;
+    Plan plan_r, plan_u;          // reduce and update kernels
+    bool staged = true;
+    Segment *d_segs_r = nullptr, *d_segs_u = nullptr;
+    int *d_first_r = nullptr, *d_first_u = nullptr;
     float *d_gbar = nullptr;
     double2 *d_partials = nullptr;
     unsigned *d_ticket = nullptr;
@@ -593,6 +926,70 @@ adascale_status cuda_fail(adascale_ctx *c, cudaError_t e, const char *what)
         cudaError_t e_ = (call);                                    \
         if (e_ != cudaSuccess) return cuda_fail(ctx, e_, #call);    \
     } while (0)
+
+// Splits the tensors over at most max_blocks blocks so that every block gets the same cost,
+// where a segment costs its length in units (one unit = `unit` elements, the width of a
+// vector access) plus a fixed `seg_cost` for staging its row pointers.  Segment boundaries
+// are multiples of `unit` elements from the tensor's start, so a 16-byte aligned tensor
+// stays 16-byte aligned in every segment.
+Plan make_plan(const std::vector<long long> &numel, const std::vector<long long> &goff, int unit,
+               long long seg_cost, int max_blocks)
+{
+    Plan p;
+    long long units_total = 0, tensors = 0;
+    for (long long n : numel)
+        if (n > 0) {
+            units_total += (n + unit - 1) / unit;
+            tensors += 1;
+        }
+    if (units_total == 0) {
+        p.n_blocks = 0;
+        p.first.assign(1, 0);
+        return p;
+    }
+    long long nb = (units_total + kMinUnitsPerBlock - 1) / kMinUnitsPerBlock;
+    if (nb > max_blocks) nb = max_blocks;
+    if (nb < 1) nb = 1;
+    // every block boundary that falls inside a tensor adds one more segment
+    const long long cost_total = units_total + seg_cost * (tensors + nb - 1);
+    const long long target = (cost_total + nb - 1) / nb;
+    p.n_blocks = (int)nb;
+    p.first.assign((size_t)nb + 1, 0);
+    long long b = 0, acc = 0;
+    for (size_t k = 0; k < numel.size(); ++k) {
+        const long long n = numel[k];
+        long long rem = n > 0 ? (n + unit - 1) / unit : 0, off = 0;
+        while (rem > 0) {
+            if (b < nb - 1 && acc > 0 && acc + seg_cost + 1 > target) {  // not worth starting here
+                p.first[(size_t)++b] = (int)p.segs.size();
+                acc = 0;
+            }
+            long long room = target - acc - seg_cost;
+            if (room < 1) room = 1;
+            const long long take = (b == nb - 1 || rem < room) ? rem : room;
+            Segment sg;
+            sg.tensor = (int)k;
+            sg.off = off * unit;
+            sg.goff = goff[k] + sg.off;
+            const long long len = (sg.off + take * unit <= n) ? take * unit : n - sg.off;
+            sg.len = (int)len;
+            p.segs.push_back(sg);
+            acc += take + seg_cost;
+            off += take;
+            rem -= take;
+        }
+    }
+    while (b < nb) p.first[(size_t)++b] = (int)p.segs.size();
+    return p;
+}
+
+// Fixed cost of one segment in units: staging S row pointers takes about as long as
+// streaming ~16 KB does at one block's share of the bandwidth, and a unit is 16*S bytes.
+long long segment_cost(int S)
+{
+    const long long c = 1024 / (S > 0 ? S : 1);
+    return c < 4 ? 4 : c;
+}
 
 double resolve_theta(const adascale_ctx *c)
 {
@@ -646,9 +1043,9 @@ adascale_status table_sync(adascale_ctx *ctx, PtrTable &t, const std::vector<u64
 }
 
 template <int DT>
-cudaError_t launch_reduce(int B, const ReduceArgs &a, size_t smem, cudaStream_t s)
+cudaError_t launch_reduce(int B, int n_blocks, const ReduceArgs &a, size_t smem, cudaStream_t s)
 {
-    const dim3 grid(a.n_chunks), block(kThreads);
+    const dim3 grid(n_blocks), block(kThreads);
     switch (B) {
     case 1: k_reduce<DT, 1><<<grid, block, smem, s>>>(a); break;
     case 2: k_reduce<DT, 2><<<grid, block, smem, s>>>(a); break;
@@ -659,6 +1056,56 @@ cudaError_t launch_reduce(int B, const ReduceArgs &a, size_t smem, cudaStream_t 
 }
 
 int batch_for(int S) { return S >= 8 ? 8 : S >= 4 ? 4 : S >= 2 ? 2 : 1; }
+
+// Columns per consumer thread: as many as keep one stage (rows x 256 x CPT elements) within 32 KB.
+int cols_per_thread(int dtype, int S)
+{
+    const int rps = S < kRowsPerStage ? S : kRowsPerStage;
+    const int budget = (dtype == ADASCALE_BF16 ? 64 : 32) / rps;
+    int cpt = 8;
+    while (cpt > budget && cpt > 1) cpt >>= 1;
+    if (dtype == ADASCALE_BF16 && cpt < 2) cpt = 2;
+    return cpt;
+}
+
+size_t staged_smem(int dtype, int S, int cpt)
+{
+    const int rps = S < kRowsPerStage ? S : kRowsPerStage;
+    return (size_t)kStages * rps * kConsumers * cpt * (dtype == ADASCALE_BF16 ? 2 : 4);
+}
+
+template <int DT, int CPT>
+cudaError_t launch_staged_one(int n_blocks, const ReduceArgs &a, size_t smem, cudaStream_t s)
+{
+    static bool configured[64] = {false};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(k_reduce_staged<DT, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)(kStages * 32 * 1024));
+        if (e != cudaSuccess) return e;
+        configured[dev] = true;
+    }
+    k_reduce_staged<DT, CPT><<<dim3(n_blocks), dim3(kStagedThreads), smem, s>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_staged(int dtype, int cpt, int n_blocks, const ReduceArgs &a, size_t smem, cudaStream_t s)
+{
+    if (dtype == ADASCALE_BF16) {
+        switch (cpt) {
+        case 2: return launch_staged_one<ADASCALE_BF16, 2>(n_blocks, a, smem, s);
+        case 4: return launch_staged_one<ADASCALE_BF16, 4>(n_blocks, a, smem, s);
+        default: return launch_staged_one<ADASCALE_BF16, 8>(n_blocks, a, smem, s);
+        }
+    }
+    switch (cpt) {
+    case 1: return launch_staged_one<ADASCALE_F32, 1>(n_blocks, a, smem, s);
+    case 2: return launch_staged_one<ADASCALE_F32, 2>(n_blocks, a, smem, s);
+    case 4: return launch_staged_one<ADASCALE_F32, 4>(n_blocks, a, smem, s);
+    default: return launch_staged_one<ADASCALE_F32, 8>(n_blocks, a, smem, s);
+    }
+}
 
 bool valid_sched(const adascale_lr_schedule *s)
 {
@@ -693,17 +1140,17 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
     }
     adascale_status st = table_sync(ctx, ctx->tg, fresh, s);
     if (st != ADASCALE_OK) return st;
-    if (ctx->n_chunks == 0) return ADASCALE_OK;
+    if (ctx->plan_r.n_blocks == 0) return ADASCALE_OK;
 
     ReduceArgs a;
-    a.chunks = ctx->d_chunks;
+    a.segs = ctx->d_segs_r;
+    a.first = ctx->d_first_r;
     a.gptr = ctx->tg.dev;
     a.gflags = reinterpret_cast<const unsigned *>(ctx->tg.dev + (size_t)ctx->max_S * T);
     a.gbar = ctx->d_gbar;
     a.partials = ctx->d_partials;
     a.ticket = ctx->d_ticket;
     a.st = ctx->d_state;
-    a.n_chunks = ctx->n_chunks;
     a.S = S;
     a.T = T;
     a.fS = (float)S;
@@ -721,8 +1168,15 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
 
     const size_t smem = (size_t)S * sizeof(u64);
     const int B = batch_for(S);
-    cudaError_t e = ctx->dtype == ADASCALE_BF16 ? launch_reduce<ADASCALE_BF16>(B, a, smem, s)
-                                                : launch_reduce<ADASCALE_F32>(B, a, smem, s);
+    const int nb = ctx->plan_r.n_blocks;
+    cudaError_t e;
+    if (ctx->staged) {
+        const int cpt = cols_per_thread(ctx->dtype, S);
+        e = launch_staged(ctx->dtype, cpt, nb, a, staged_smem(ctx->dtype, S, cpt), s);
+    } else {
+        e = ctx->dtype == ADASCALE_BF16 ? launch_reduce<ADASCALE_BF16>(B, nb, a, smem, s)
+                                        : launch_reduce<ADASCALE_F32>(B, nb, a, smem, s);
+    }
     if (e != cudaSuccess) return cuda_fail(ctx, e, "launch of the reduce kernel");
     ctx->launches += 1;
     ctx->reduced = true;
@@ -747,19 +1201,19 @@ adascale_status do_update(adascale_ctx *ctx, void *const *params, void *const *m
     }
     adascale_status st = table_sync(ctx, ctx->tw, fresh, s);
     if (st != ADASCALE_OK) return st;
-    if (ctx->n_chunks == 0) return ADASCALE_OK;
+    if (ctx->plan_u.n_blocks == 0) return ADASCALE_OK;
 
     UpdateArgs a;
-    a.chunks = ctx->d_chunks;
+    a.segs = ctx->d_segs_u;
+    a.first = ctx->d_first_u;
     a.wv = ctx->tw.dev;
     a.wflags = reinterpret_cast<const unsigned *>(ctx->tw.dev + (size_t)2 * T);
     a.gbar = ctx->d_gbar;
     a.st = ctx->d_state;
-    a.n_chunks = ctx->n_chunks;
     a.T = T;
     a.rho = (float)ctx->rho;
     a.lambda = (float)ctx->lambda;
-    k_update<<<dim3(ctx->n_chunks), dim3(kThreads), 0, s>>>(a);
+    k_update<<<dim3(ctx->plan_u.n_blocks), dim3(kThreads), 0, s>>>(a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(ctx, e, "launch of the update kernel");
     ctx->launches += 1;
@@ -783,7 +1237,7 @@ void fill_stats(const adascale_ctx *ctx, const DevState &d, adascale_stats *o)
     o->t = d.t;
     o->n_samples = d.n;
     o->skipped = d.skipped;
-    o->status_bits = d.status;
+    o->status_bits = d.status | d.fault;
     (void)ctx;
 }
 
@@ -807,6 +1261,31 @@ const char *adascale_strerror(adascale_status s)
 const char *adascale_last_error(const adascale_ctx *ctx) { return ctx ? ctx->err.c_str() : ""; }
 
 int64_t adascale_launch_count(const adascale_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+int64_t adascale_plan(const int64_t *numel, int32_t n_tensors, int32_t unit, int64_t seg_cost,
+                      int32_t max_blocks, int64_t *out, int64_t cap)
+{
+    if (!numel || n_tensors < 1 || unit < 1 || seg_cost < 0 || max_blocks < 1 || cap < 0 || (cap > 0 && !out))
+        return -1;
+    std::vector<long long> n(numel, numel + n_tensors), goff;
+    long long g = 0;
+    for (long long x : n) {
+        if (x < 0) return -1;
+        goff.push_back(g);
+        g += (x + kGbarAlign - 1) / kGbarAlign * kGbarAlign;
+    }
+    const Plan p = make_plan(n, goff, unit, seg_cost, max_blocks);
+    int64_t written = 0;
+    for (int b = 0; b < p.n_blocks; ++b)
+        for (int i = p.first[b]; i < p.first[b + 1]; ++i, ++written)
+            if (written < cap) {
+                out[4 * written + 0] = p.segs[i].tensor;
+                out[4 * written + 1] = p.segs[i].off;
+                out[4 * written + 2] = p.segs[i].len;
+                out[4 * written + 3] = b;
+            }
+    return (int64_t)p.segs.size();
+}
 
 adascale_status adascale_init(const adascale_config *cfg, adascale_ctx **out)
 {
@@ -838,43 +1317,44 @@ adascale_status adascale_init(const adascale_config *cfg, adascale_ctx **out)
     ctx->flags = cfg->flags;
     ctx->numel.assign(cfg->numel, cfg->numel + cfg->n_tensors);
 
-    // chunk table: every tensor is cut into blocks of kChunk elements; chunk boundaries are
-    // multiples of 8 elements so a 16-byte aligned tensor stays 16-byte aligned in every chunk
-    const int chunk = ctx->dtype == ADASCALE_BF16 ? kChunkBF16 : kChunkF32;
-    std::vector<Chunk> chunks;
     long long g = 0;
     for (int k = 0; k < ctx->T; ++k) {
         ctx->goff.push_back(g);
         const long long n = ctx->numel[k];
-        for (long long o = 0; o < n; o += chunk) {
-            Chunk c;
-            c.off = o;
-            c.goff = g + o;
-            c.tensor = k;
-            c.len = (int)((n - o) < chunk ? (n - o) : chunk);
-            chunks.push_back(c);
-        }
         ctx->P += n;
         g += (n + kGbarAlign - 1) / kGbarAlign * kGbarAlign;
     }
     ctx->gbar_elems = g;
-    if (chunks.size() > 0x7fffffffull) {
-        delete ctx;
-        return ADASCALE_ERR_TOO_LARGE;
-    }
-    ctx->n_chunks = (int)chunks.size();
 
     DeviceGuard guard(ctx->device);
     adascale_status rc = ADASCALE_OK;
     auto body = [&]() -> adascale_status {
         if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
-        const size_t nc = chunks.empty() ? 1 : chunks.size();
-        CU(cudaMalloc(&ctx->d_chunks, nc * sizeof(Chunk)));
-        if (!chunks.empty())
-            CU(cudaMemcpy(ctx->d_chunks, chunks.data(), chunks.size() * sizeof(Chunk), cudaMemcpyHostToDevice));
+        int sms = 0;
+        CU(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device));
+        // one plan per kernel: the grid is sized to the device, the split is fixed from here on,
+        // which is what makes the fixed-order sums reproducible from run to run
+        ctx->staged = std::getenv("ADASCALE_REDUCE_LDG") == nullptr;
+        ctx->plan_r = make_plan(ctx->numel, ctx->goff, 8, segment_cost(ctx->S),
+                                sms * (ctx->staged ? 2 : kReduceBlocksPerSM));
+        ctx->plan_u = make_plan(ctx->numel, ctx->goff, 4, 64, sms * kUpdateBlocksPerSM);
+        if (ctx->plan_r.segs.size() > 0x7fffffffull) return ADASCALE_ERR_TOO_LARGE;
+        auto upload = [&](const Plan &pl, Segment **dsegs, int **dfirst) -> adascale_status {
+            const size_t ns = pl.segs.empty() ? 1 : pl.segs.size();
+            CU(cudaMalloc(dsegs, ns * sizeof(Segment)));
+            CU(cudaMalloc(dfirst, pl.first.size() * sizeof(int)));
+            if (!pl.segs.empty())
+                CU(cudaMemcpy(*dsegs, pl.segs.data(), pl.segs.size() * sizeof(Segment), cudaMemcpyHostToDevice));
+            CU(cudaMemcpy(*dfirst, pl.first.data(), pl.first.size() * sizeof(int), cudaMemcpyHostToDevice));
+            return ADASCALE_OK;
+        };
+        adascale_status s0 = upload(ctx->plan_r, &ctx->d_segs_r, &ctx->d_first_r);
+        if (s0 != ADASCALE_OK) return s0;
+        s0 = upload(ctx->plan_u, &ctx->d_segs_u, &ctx->d_first_u);
+        if (s0 != ADASCALE_OK) return s0;
         CU(cudaMalloc(&ctx->d_gbar, (size_t)(g > 0 ? g : 1) * sizeof(float)));
         CU(cudaMemset(ctx->d_gbar, 0, (size_t)(g > 0 ? g : 1) * sizeof(float)));
-        CU(cudaMalloc(&ctx->d_partials, nc * sizeof(double2)));
+        CU(cudaMalloc(&ctx->d_partials, (size_t)(ctx->plan_r.n_blocks + 1) * sizeof(double2)));
         CU(cudaMalloc(&ctx->d_ticket, sizeof(unsigned)));
         CU(cudaMemset(ctx->d_ticket, 0, sizeof(unsigned)));
         CU(cudaMalloc(&ctx->d_state, sizeof(DevState)));
@@ -887,7 +1367,6 @@ adascale_status adascale_init(const adascale_config *cfg, adascale_ctx **out)
         CU(cudaMallocHost(&ctx->h_snap, sizeof(DevState)));
         std::memset(ctx->h_snap, 0, sizeof(DevState));
         CU(cudaEventCreateWithFlags(&ctx->ev_snap, cudaEventDisableTiming));
-        // dynamic shared memory of the reduce kernel: S row pointers (32 KB at the maximum S)
         return ADASCALE_OK;
     };
     rc = body();
@@ -905,7 +1384,10 @@ adascale_status adascale_destroy(adascale_ctx *ctx)
     DeviceGuard guard(ctx->device);
     if (guard.ok) {
         cudaDeviceSynchronize();
-        cudaFree(ctx->d_chunks);
+        cudaFree(ctx->d_segs_r);
+        cudaFree(ctx->d_segs_u);
+        cudaFree(ctx->d_first_r);
+        cudaFree(ctx->d_first_u);
         cudaFree(ctx->d_gbar);
         cudaFree(ctx->d_partials);
         cudaFree(ctx->d_ticket);
