@@ -213,15 +213,18 @@ adascale_status adascale_step_host(adascale_ctx *ctx, const void *const *grads, 
 adascale_status adascale_stream_probe(int32_t kind, void *a, void *b, int64_t n_bytes, void *cuda_stream);
 
 /*
- * Host-only view of how the library splits a tensor list over the blocks of its persistent
- * kernels (no counterpart in the paper; used by tests).  numel: host array [n_tensors];
- * unit: elements per vector access; seg_cost: fixed cost of a segment in units;
- * max_blocks: grid size.  Writes up to cap rows of 4 int64 {tensor, first element, length
- * in elements, block} into out, in block order, and returns the number of segments
- * (which may exceed cap), or -1 for invalid arguments.  Makes no CUDA call.
+ * Host-only view of how the reduce kernel tiles a tensor list (no counterpart in the paper;
+ * used by tests and for sizing).  numel: host array [n_tensors]; aligned: host array
+ * [n_tensors], non-zero where all S gradient pointers of the tensor are 16-byte aligned
+ * (NULL = all aligned); n_blocks: grid size the tiling is tuned for.  Writes the number of
+ * staged tiles before each tensor into tprefix[0..n_tensors] and of scalar-path tiles into
+ * sprefix[0..n_tensors], the columns of one staged tile into *tile_cols and the rows of one
+ * shared-memory stage into *rows.  Tile t is processed by block t mod gridDim.  Makes no
+ * CUDA call.  Errors: INVALID_ARG.
  */
-int64_t adascale_plan(const int64_t *numel, int32_t n_tensors, int32_t unit, int64_t seg_cost,
-                      int32_t max_blocks, int64_t *out, int64_t cap);
+adascale_status adascale_tiling(const int64_t *numel, int32_t n_tensors, int32_t grad_dtype, int32_t S,
+                                const uint8_t *aligned, int32_t n_blocks, int64_t *tprefix, int64_t *sprefix,
+                                int32_t *tile_cols, int32_t *rows);
 
 /* Number of kernels the library has launched through this context since init. */
 int64_t adascale_launch_count(const adascale_ctx *ctx);

@@ -22,7 +22,7 @@ STATE_BYTES = 128
 
 EXPORTS = ("adascale_init", "adascale_step", "adascale_reduce", "adascale_update", "adascale_get_gain_tau",
            "adascale_mean_grad", "adascale_set_scale", "adascale_get_state", "adascale_set_state",
-           "adascale_step_host", "adascale_stream_probe", "adascale_plan", "adascale_launch_count",
+           "adascale_step_host", "adascale_stream_probe", "adascale_tiling", "adascale_launch_count",
            "adascale_destroy",
            "adascale_strerror", "adascale_last_error")
 
@@ -72,9 +72,9 @@ def _load():
     L.adascale_set_state.argtypes = [vp, vp]
     L.adascale_step_host.argtypes = [vp, vpp, vpp, vpp, C.POINTER(LrSchedule), C.POINTER(Stats), vp]
     L.adascale_stream_probe.argtypes = [C.c_int32, vp, vp, C.c_int64, vp]
-    L.adascale_plan.argtypes = [C.POINTER(C.c_int64), C.c_int32, C.c_int32, C.c_int64, C.c_int32,
-                                C.POINTER(C.c_int64), C.c_int64]
-    L.adascale_plan.restype = C.c_int64
+    L.adascale_tiling.argtypes = [C.POINTER(C.c_int64), C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_uint8),
+                                  C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int32),
+                                  C.POINTER(C.c_int32)]
     L.adascale_launch_count.argtypes = [vp]
     L.adascale_launch_count.restype = C.c_int64
     L.adascale_destroy.argtypes = [vp]
@@ -83,7 +83,7 @@ def _load():
     L.adascale_last_error.argtypes = [vp]
     L.adascale_last_error.restype = C.c_char_p
     for name in EXPORTS:
-        if name not in ("adascale_launch_count", "adascale_strerror", "adascale_last_error", "adascale_plan"):
+        if name not in ("adascale_launch_count", "adascale_strerror", "adascale_last_error"):
             getattr(L, name).restype = C.c_int
     return L
 
@@ -240,15 +240,18 @@ class AdaScale:
         return int(lib.adascale_launch_count(self._ctx))
 
 
-def plan(numels, unit, seg_cost, max_blocks):
-    """Rows (tensor, first element, length, block) of the static split; host only."""
-    arr = (C.c_int64 * len(numels))(*[int(n) for n in numels])
-    n = lib.adascale_plan(arr, len(numels), int(unit), int(seg_cost), int(max_blocks), None, 0)
-    if n < 0:
-        raise ValueError("invalid plan arguments")
-    out = (C.c_int64 * (4 * max(n, 1)))()
-    lib.adascale_plan(arr, len(numels), int(unit), int(seg_cost), int(max_blocks), out, n)
-    return [tuple(out[4 * i:4 * i + 4]) for i in range(n)]
+def tiling(numels, S, grad_dtype="f32", aligned=None, n_blocks=296):
+    """Host-only: (staged-tile prefix, scalar-tile prefix, tile columns, rows per stage)."""
+    T = len(numels)
+    arr = (C.c_int64 * T)(*[int(n) for n in numels])
+    al = None if aligned is None else (C.c_uint8 * T)(*[1 if a else 0 for a in aligned])
+    tp, sp = (C.c_int64 * (T + 1))(), (C.c_int64 * (T + 1))()
+    cols, rows = C.c_int32(), C.c_int32()
+    status = lib.adascale_tiling(arr, T, {"f32": F32, "bf16": BF16}.get(grad_dtype, grad_dtype), int(S), al,
+                                 int(n_blocks), tp, sp, C.byref(cols), C.byref(rows))
+    if status != OK:
+        raise AdaScaleError(status, strerror(status))
+    return list(tp), list(sp), cols.value, rows.value
 
 
 def stream_probe(kind, a, b, n_bytes, stream=None, device=0):

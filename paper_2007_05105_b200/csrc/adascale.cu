@@ -1,13 +1,19 @@
 // AdaScale SGD gain-ratio step for sm_100a: kernels and the C-ABI host glue.
 //
-// Three kernels make up one iteration (paper: Sec. 3.2, App. B.3, Eq. 2-3):
-//   reduce  - streams the S x P gradient matrix once, writes the mean gradient and one
-//             pair (sum of squared deviations, squared norm of the mean) per block; the
-//             block that finishes last adds the pairs in index order and runs the scalar
-//             part (estimates, clamps, moving averages, r_t, eta_t, tau_{t+1}).
+// Two kernels make up one iteration (paper: Sec. 3.2, App. B.3, Eq. 2-3):
+//   reduce  - streams the S x P gradient matrix once through shared memory (bulk asynchronous
+//             copies completed on mbarriers, a producer warp and eight consumer warps), writes
+//             the mean gradient and one pair (sum of squared deviations, squared norm of the
+//             mean) per block; the block that finishes last adds the pairs in index order and
+//             runs the scalar part (estimates, clamps, moving averages, r_t, eta_t, tau_{t+1}).
 //   update  - v <- rho v + (gbar + lambda w), w <- w - eta_t v, reading eta_t from the device.
-//   probes  - trivial streaming kernels that calibrate the bandwidth ceiling.
+// Three trivial streaming kernels calibrate the bandwidth ceiling.
 // The path is bound by HBM bandwidth; there is no contraction, hence no tensor-core work.
+//
+// Work distribution: every tensor is cut into tiles; tile t belongs to block t mod gridDim.
+// All blocks therefore advance through each gradient row as one front, which keeps DRAM
+// pages hot, and the split does not depend on how the hardware schedules blocks, so the
+// fixed-order sums are reproducible from run to run.
 #include "../../include/adascale.h"
 
 #include <cuda_runtime.h>
@@ -22,32 +28,23 @@
 
 namespace {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 256;             // consumer threads of the reduce kernel, all threads of the update kernel
 constexpr int kWarps = kThreads / 32;
-constexpr int kReduceBlocksPerSM = 4;  // resident blocks the reduce kernel is compiled for
-constexpr int kUpdateBlocksPerSM = 8;  // same for the update kernel
-constexpr int kMinUnitsPerBlock = 512; // do not spread a small job over more blocks than this allows
-constexpr int kGbarAlign = 64;    // every tensor's mean gradient starts on a 256-byte boundary
-constexpr int kRing = 4;          // pinned staging slots for pointer-table uploads
+constexpr int kStagedThreads = kThreads + 32;  // + 1 producer warp
+constexpr int kStagedWarps = kStagedThreads / 32;
+constexpr int kStages = 3;                // shared-memory stages per block
+constexpr int kMaxRowsPerStage = 16;      // rows of one stage; larger S goes through in row chunks
+constexpr int kStageBytes = 32 * 1024;    // upper bound of one stage
+constexpr int kReduceBlocksPerSM = 2;
+constexpr int kUpdateBlocksPerSM = 8;
+constexpr int kScalarTile = 2048;         // elements per tile on the unaligned / ragged-tail path
+constexpr int kUpdateTile = 1024;         // elements per tile of the update kernel: one 128-bit access per thread
+constexpr int kGbarAlign = 64;            // every tensor's mean gradient starts on a 256-byte boundary
+constexpr int kRing = 4;                  // pinned staging slots for pointer-table uploads
 constexpr int kMaxS = 4096;
+constexpr unsigned kSpinLimit = 1u << 22; // bounded waits: give up, flag, leave
 
 typedef unsigned long long u64;
-
-// A contiguous run of elements of one tensor, owned by one block.
-struct Segment {
-    long long off;   // first element inside the tensor
-    long long goff;  // first element inside the mean-gradient workspace
-    int tensor;
-    int len;         // elements
-};
-
-// Static split of all tensors over the blocks of a persistent grid: block b owns
-// segs[first[b]] .. segs[first[b+1]-1].  Built once on the host (see make_plan).
-struct Plan {
-    std::vector<Segment> segs;
-    std::vector<int> first;  // n_blocks + 1 entries
-    int n_blocks = 0;
-};
 
 // Scalar state kept on the device between iterations.
 struct DevState {
@@ -65,7 +62,7 @@ struct DevState {
 };
 
 struct ScalarCfg {
-    double eps, theta;  // theta already resolved (paper rule applied on the host side of set_scale)
+    double eps, theta;  // theta already resolved on the host (the paper's rule follows S)
     unsigned flags;
     int S;
 };
@@ -76,11 +73,17 @@ struct Sched {
     double w[ADASCALE_MAX_MILESTONES];
 };
 
+// Tiling of the tensor list for one launch of the reduce kernel.  A tensor whose S row
+// pointers are 16-byte aligned contributes ceil(cols / tile_cols) staged tiles for its first
+// cols = numel & ~7 elements and one scalar tile for the ragged rest; any other tensor
+// contributes only scalar tiles of kScalarTile elements.
 struct ReduceArgs {
-    const Segment *segs;
-    const int *first;
-    const u64 *gptr;        // [S * T] row pointers
-    const unsigned *gflags; // [T] bit0: all S rows of the tensor are 16-byte aligned
+    const u64 *gptr;          // [S * T] row pointers
+    const long long *tprefix; // [T + 1] staged tiles before tensor k
+    const long long *sprefix; // [T + 1] scalar tiles before tensor k
+    const unsigned *gflags;   // [T] bit0: all S rows of the tensor are 16-byte aligned
+    const long long *numel;   // [T]
+    const long long *goff;    // [T] offset of the tensor in the mean-gradient workspace
     float *gbar;
     double2 *partials;
     unsigned *ticket;
@@ -92,10 +95,11 @@ struct ReduceArgs {
 };
 
 struct UpdateArgs {
-    const Segment *segs;
-    const int *first;
-    const u64 *wv;          // [2 * T]: parameters then momentum
-    const unsigned *wflags; // [T] bit0: both pointers 16-byte aligned
+    const u64 *wv;            // [2 * T]: parameters then momentum
+    const unsigned *wflags;   // [T] bit0: both pointers 16-byte aligned
+    const long long *uprefix; // [T + 1] update tiles before tensor k
+    const long long *numel;
+    const long long *goff;
     const float *gbar;
     const DevState *st;
     int T;
@@ -147,22 +151,7 @@ template <> struct Elem<ADASCALE_BF16> {
     }
 };
 
-// ---------------------------------------------------------------------------------------
-// One column vector (4 fp32 or 8 bf16 columns) of all S rows.
-//
-// Per column the S values are shifted by a value c taken from the data:  d_i = g_i - c.
-// With s1 = sum d_i and s2 = sum d_i^2 the mean is c + s1/S and the summed squared
-// deviation is s2 - s1^2/S.  Because c is itself (close to) a sample, the subtraction
-// loses a factor of order S at worst, not the |mean|^2/sigma^2 that the raw formula of
-// App. B.3 loses; identical rows give exactly zero; and every row is consumed as it
-// arrives, so no register array of S rows is needed.
-//   - c is the median of the first three rows (row 0 when fewer than four rows are
-//     fetched together): one outlier among them cannot become the shift, which keeps
-//     |s1| and with it the rounding error of the mean small under heavy-tailed noise.
-//   - s1 is summed in blocks of B rows (a fresh partial per block, then one add), so the
-//     long chain of roundings happens on small partial sums.
-// B <= S rows are requested together to keep 16*B bytes per thread in flight.
-// ---------------------------------------------------------------------------------------
+// d = x - c, blocked first moment, running second moment, for V columns of one row.
 template <int V>
 __device__ __forceinline__ void accumulate_row(const float *x, const float *c, float *p1, float *s2)
 {
@@ -174,116 +163,10 @@ __device__ __forceinline__ void accumulate_row(const float *x, const float *c, f
     }
 }
 
-template <int DT, int B>
-__device__ __forceinline__ void column_vector(const u64 *rowp, size_t boff, int S, float invS, float fS,
-                                              float *gb, float &dsum, float &nsum)
-{
-    constexpr int V = Elem<DT>::kVec;
-    float c[V], s1[V], s2[V], p1[V], x[V];
-#pragma unroll
-    for (int k = 0; k < V; ++k) s1[k] = s2[k] = p1[k] = 0.f;
-
-    uint4 q[B];
-#pragma unroll
-    for (int b = 0; b < B; ++b) q[b] = ld_stream16((const char *)rowp[b] + boff);
-    if (B >= 4) {
-        float x1[V], x2[V];
-        Elem<DT>::unpack(q[0], x);
-        Elem<DT>::unpack(q[1], x1);
-        Elem<DT>::unpack(q[2], x2);
-#pragma unroll
-        for (int k = 0; k < V; ++k) {
-            const float lo = fminf(x[k], x1[k]), hi = fmaxf(x[k], x1[k]);
-            c[k] = fmaxf(lo, fminf(hi, x2[k]));  // median of three
-        }
-        accumulate_row<V>(x, c, p1, s2);
-        accumulate_row<V>(x1, c, p1, s2);
-        accumulate_row<V>(x2, c, p1, s2);
-#pragma unroll
-        for (int b = 3; b < B; ++b) {
-            Elem<DT>::unpack(q[b], x);
-            accumulate_row<V>(x, c, p1, s2);
-        }
-    } else {
-        Elem<DT>::unpack(q[0], c);  // d_0 = 0
-#pragma unroll
-        for (int b = 1; b < B; ++b) {
-            Elem<DT>::unpack(q[b], x);
-            accumulate_row<V>(x, c, p1, s2);
-        }
-    }
-#pragma unroll
-    for (int k = 0; k < V; ++k) s1[k] = p1[k];
-
-    int i = B;
-    for (; i + B <= S; i += B) {
-#pragma unroll
-        for (int b = 0; b < B; ++b) q[b] = ld_stream16((const char *)rowp[i + b] + boff);
-#pragma unroll
-        for (int k = 0; k < V; ++k) p1[k] = 0.f;
-#pragma unroll
-        for (int b = 0; b < B; ++b) {
-            Elem<DT>::unpack(q[b], x);
-            accumulate_row<V>(x, c, p1, s2);
-        }
-#pragma unroll
-        for (int k = 0; k < V; ++k) s1[k] += p1[k];
-    }
-    if (i < S) {
-#pragma unroll
-        for (int k = 0; k < V; ++k) p1[k] = 0.f;
-        for (; i < S; ++i) {
-            q[0] = ld_stream16((const char *)rowp[i] + boff);
-            Elem<DT>::unpack(q[0], x);
-            accumulate_row<V>(x, c, p1, s2);
-        }
-#pragma unroll
-        for (int k = 0; k < V; ++k) s1[k] += p1[k];
-    }
-
-    float m[V];
-    float dacc = 0.f, nacc = 0.f;
-#pragma unroll
-    for (int k = 0; k < V; ++k) {
-        // quotient s1/S: reciprocal multiply plus one residual correction (1/S is not exact
-        // unless S is a power of two, and a biased 1/S would bias every column the same way)
-        float qk = s1[k] * invS;
-        const float res = fmaf(-qk, fS, s1[k]);
-        qk = fmaf(res, invS, qk);
-        m[k] = c[k] + qk;
-        dacc += fmaf(-qk, s1[k], s2[k]);
-        nacc = fmaf(m[k], m[k], nacc);
-    }
-#pragma unroll
-    for (int k = 0; k < V; k += 4) *(float4 *)(gb + k) = make_float4(m[k], m[k + 1], m[k + 2], m[k + 3]);
-    dsum = dacc;
-    nsum = nacc;
-}
-
-// One column, any alignment, any S: plain two-pass with the residual correction of the mean.
+// One column, any alignment, any S: plain two-pass with a residual correction of the mean.
+// Row pointers come straight from the device table.
 template <int DT>
-__device__ __forceinline__ void column_scalar(const u64 *rowp, size_t boff, int S, float fS, float *gb,
-                                              float &dsum, float &nsum)
-{
-    float sum = 0.f;
-    for (int i = 0; i < S; ++i) sum += Elem<DT>::load1((const char *)rowp[i] + boff);
-    float m0 = sum / fS;
-    float e = 0.f, qq = 0.f;
-    for (int i = 0; i < S; ++i) {
-        float d = Elem<DT>::load1((const char *)rowp[i] + boff) - m0;
-        e += d;
-        qq = fmaf(d, d, qq);
-    }
-    float corr = e / fS;
-    float m = m0 + corr;
-    *gb = m;
-    dsum = fmaf(-corr, e, qq);
-    nsum = m * m;
-}
-
-// Same, with the row pointers read from the device table instead of shared memory.
-template <int DT>
-__device__ __forceinline__ void column_scalar_direct(const u64 *gptr, int T, int tensor, size_t boff, int S,
+__device__ __forceinline__ void column_scalar(const u64 *gptr, int T, int tensor, size_t boff, int S,
                                                      float fS, float *gb, float &dsum, float &nsum)
 {
     float sum = 0.f;
@@ -411,90 +294,6 @@ __device__ void scalar_step(DevState *st, const ScalarCfg &c, const Sched &sched
 
 // Persistent grid: every block walks its own segments and keeps two fp64 accumulators per
 // thread for the whole launch, so there is one block reduction and one partial pair per block.
-template <int DT, int B>
-__global__ void __launch_bounds__(kThreads, kReduceBlocksPerSM) k_reduce(const __grid_constant__ ReduceArgs a)
-{
-    extern __shared__ u64 rowp[];
-    __shared__ double sa[kWarps], sb[kWarps];
-    __shared__ bool is_last;
-
-    constexpr int V = Elem<DT>::kVec;
-    constexpr int E = Elem<DT>::kBytes;
-    const int tid = threadIdx.x;
-    double accD = 0.0, accN = 0.0;
-
-    const int seg_end = a.first[blockIdx.x + 1];
-    for (int sidx = a.first[blockIdx.x]; sidx < seg_end; ++sidx) {
-        const Segment sg = a.segs[sidx];
-        __syncthreads();  // the previous segment's row pointers are no longer needed
-        for (int i = tid; i < a.S; i += kThreads)
-            rowp[i] = a.gptr[(size_t)i * a.T + sg.tensor] + (u64)sg.off * E;
-        __syncthreads();
-
-        float *gb = a.gbar + sg.goff;
-        int first_scalar = 0;
-        if (a.gflags[sg.tensor] & 1u) {
-            const int nv = sg.len / V;
-            for (int v = tid; v < nv; v += kThreads) {
-                float d, n;
-                column_vector<DT, B>(rowp, (size_t)v * 16, a.S, a.invS, a.fS, gb + (size_t)v * V, d, n);
-                accD += (double)d;
-                accN += (double)n;
-            }
-            first_scalar = nv * V;
-        }
-        for (int e = first_scalar + tid; e < sg.len; e += kThreads) {
-            float d, n;
-            column_scalar<DT>(rowp, (size_t)e * E, a.S, a.fS, gb + e, d, n);
-            accD += (double)d;
-            accN += (double)n;
-        }
-    }
-
-    block_sum2(accD, accN, sa, sb);
-    if (tid == 0) {
-        a.partials[blockIdx.x] = make_double2(accD, accN);
-        __threadfence();
-        const unsigned tk = atomicAdd(a.ticket, 1u);
-        is_last = (tk == gridDim.x - 1);
-    }
-    __syncthreads();
-    if (!is_last) return;
-
-    // Second stage, fixed order: thread j adds partials j, j+256, ... in index order, then the
-    // same block tree.  The result depends on the plan only, not on how blocks were scheduled.
-    __threadfence();
-    double d = 0.0, n = 0.0;
-    for (int i = tid; i < (int)gridDim.x; i += kThreads) {
-        const double2 p = __ldcg(&a.partials[i]);
-        d += p.x;
-        n += p.y;
-    }
-    block_sum2(d, n, sa, sb);
-    if (tid == 0) {
-        scalar_step(a.st, a.sc, a.sched, d, n);
-        *a.ticket = 0u;
-    }
-}
-
-// ---------------------------------------------------------------------------------------
-// Reduce kernel, staged variant: a producer warp streams tiles of the gradient matrix into
-// shared memory with bulk asynchronous copies (one copy per row per tile, completion counted
-// on an mbarrier), eight consumer warps read the tiles back from shared memory.  Memory
-// latency is covered by the stages in flight instead of by registers, and the consumers
-// issue no global loads or address arithmetic at all.
-//
-// A work item is (segment, column tile, row chunk): kTileThreads * CPT columns of up to
-// kRowsPerStage rows.  Row chunks let any S through: the per-column sums carry over from one
-// chunk of rows to the next and are closed after the last.
-// ---------------------------------------------------------------------------------------
-constexpr int kStages = 3;
-constexpr int kRowsPerStage = 32;
-constexpr int kConsumers = kThreads;          // 8 consumer warps
-constexpr int kStagedThreads = kThreads + 32; // + 1 producer warp
-constexpr int kStagedWarps = kStagedThreads / 32;
-constexpr unsigned kSpinLimit = 1u << 22;     // bounded waits: give up, flag, leave
-
 __device__ __forceinline__ unsigned smem_u32(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(u64 *bar, unsigned count)
@@ -583,8 +382,32 @@ __device__ __forceinline__ void store_cols(float *g, const float *m)
     }
 }
 
+
+// ---------------------------------------------------------------------------------------
+// Reduce kernel.
+//
+// Per column the S values are shifted by a value c taken from the data:  d_i = g_i - c.
+// With s1 = sum d_i and s2 = sum d_i^2 the mean is c + s1/S and the summed squared
+// deviation is s2 - s1^2/S.  Because c is (close to) a sample, the subtraction loses a
+// factor of order S at worst, not the |mean|^2/sigma^2 that the raw formula of App. B.3
+// loses; identical rows give exactly zero; and each row is consumed as it is read.
+//   - c is the median of the first three rows (row 0 when S < 3): one outlier among them
+//     cannot become the shift, which keeps |s1|, and with it the rounding error of the
+//     mean, small under heavy-tailed noise.
+//   - s1 is summed in blocks of 8 rows (a fresh partial per block, then one add), so the
+//     long chain of roundings happens on small partial sums.
+//   - per-column results enter fp64 accumulators; warp shuffles, a block tree and a
+//     fixed-order second stage do the rest in fp64.
+//
+// A producer warp streams tiles into shared memory with bulk asynchronous copies (one copy
+// per row, completion counted on an mbarrier); eight consumer warps read them back.  Memory
+// latency is covered by the stages in flight rather than by registers, and the consumers
+// issue no global loads or address arithmetic.  A work item is (tile, row chunk):
+// kThreads * CPT columns of up to kMaxRowsPerStage rows.  Row chunks let any S through: the
+// per-column sums carry over from one chunk of rows to the next and close after the last.
+// ---------------------------------------------------------------------------------------
 template <int DT, int CPT>
-__global__ void __launch_bounds__(kStagedThreads, 2) k_reduce_staged(const __grid_constant__ ReduceArgs a)
+__global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(const __grid_constant__ ReduceArgs a)
 {
     extern __shared__ __align__(128) unsigned char stage_mem[];
     __shared__ __align__(8) u64 full_bar[kStages], empty_bar[kStages];
@@ -593,19 +416,20 @@ __global__ void __launch_bounds__(kStagedThreads, 2) k_reduce_staged(const __gri
     __shared__ int abort_flag;
 
     constexpr int E = Elem<DT>::kBytes;
-    constexpr int kTile = kConsumers * CPT;     // columns per tile
-    constexpr int kRowBytes = kTile * E;        // one row of a stage
+    constexpr int kTile = kThreads * CPT;  // columns per tile
+    constexpr int kRowBytes = kTile * E;   // one row of a stage
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const bool producer = warp == kStagedWarps - 1;
-    const int S = a.S;
-    const int rps = S < kRowsPerStage ? S : kRowsPerStage;  // rows per stage
+    const int S = a.S, T = a.T;
+    const int rps = S < kMaxRowsPerStage ? S : kMaxRowsPerStage;  // rows per stage
     const int n_chunks = (S + rps - 1) / rps;
     const unsigned stage_bytes = (unsigned)rps * kRowBytes;
+    const long long n_tiles = a.tprefix[T];
 
     if (tid == 0) {
         for (int i = 0; i < kStages; ++i) {
             mbar_init(&full_bar[i], 1);
-            mbar_init(&empty_bar[i], kConsumers / 32);
+            mbar_init(&empty_bar[i], kWarps);
         }
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -616,7 +440,7 @@ __global__ void __launch_bounds__(kStagedThreads, 2) k_reduce_staged(const __gri
     double accD = 0.0, accN = 0.0;
     unsigned item = 0;  // running count of staged work items, identical in every thread
     bool timed_out = false;
-    const int seg_end = a.first[blockIdx.x + 1];
+    int k = 0;          // tensor that holds the current tile; tiles only move forward
 
     if (producer) {
         u64 policy;
@@ -624,27 +448,38 @@ __global__ void __launch_bounds__(kStagedThreads, 2) k_reduce_staged(const __gri
         int last_use[kStages];
 #pragma unroll
         for (int i = 0; i < kStages; ++i) last_use[i] = -1;
-        for (int sidx = a.first[blockIdx.x]; sidx < seg_end && !timed_out; ++sidx) {
-            const Segment sg = a.segs[sidx];
-            if (!(a.gflags[sg.tensor] & 1u)) continue;  // consumers take unaligned tensors from global memory
-            const int cols = sg.len & ~7;
-            for (int c0 = 0; c0 < cols && !timed_out; c0 += kTile) {
-                const int tc = cols - c0 < kTile ? cols - c0 : kTile;
-                for (int ch = 0; ch < n_chunks; ++ch, ++item) {
-                    const int st = item % kStages;
-                    const unsigned use = item / kStages;
-                    if (!mbar_wait(&empty_bar[st], (use & 1u) ^ 1u)) { timed_out = true; break; }
-                    const int r0 = ch * rps;
-                    const int rows = S - r0 < rps ? S - r0 : rps;
-                    if (lane == 0) mbar_expect_tx(&full_bar[st], (unsigned)rows * tc * E);
-                    __syncwarp();
+        int held = -1;      // tensor whose row pointer this lane holds (row = lane, when S <= 32)
+        const char *rowptr = nullptr;
+        for (long long t = blockIdx.x; t < n_tiles && !timed_out; t += gridDim.x) {
+            while (t >= a.tprefix[k + 1]) ++k;
+            const long long c0 = (t - a.tprefix[k]) * kTile;
+            const long long cols = a.numel[k] & ~7LL;
+            const int tc = cols - c0 < kTile ? (int)(cols - c0) : kTile;
+            if (held != k) {
+                held = k;
+                if (lane < S) rowptr = (const char *)a.gptr[(size_t)lane * T + k];
+            }
+            for (int ch = 0; ch < n_chunks; ++ch, ++item) {
+                const int st = item % kStages;
+                const unsigned use = item / kStages;
+                if (!mbar_wait(&empty_bar[st], (use & 1u) ^ 1u)) { timed_out = true; break; }
+                const int r0 = ch * rps;
+                const int rows = S - r0 < rps ? S - r0 : rps;
+                if (lane == 0) mbar_expect_tx(&full_bar[st], (unsigned)rows * tc * E);
+                __syncwarp();
 #pragma unroll
-                    for (int i = 0; i < kStages; ++i)
-                        if (i == st) last_use[i] = (int)use;
+                for (int i = 0; i < kStages; ++i)
+                    if (i == st) last_use[i] = (int)use;
+                unsigned char *dst = stage_mem + (size_t)st * stage_bytes;
+                if (r0 + rps <= 32) {
+                    // rows r0 .. r0+rows-1 live in lanes r0 .. : each lane copies its own row
+                    const int r = lane - r0;
+                    if (r >= 0 && r < rows)
+                        bulk_load(dst + (size_t)r * kRowBytes, rowptr + (size_t)c0 * E, (unsigned)tc * E, &full_bar[st], policy);
+                } else {
                     for (int r = lane; r < rows; r += 32) {
-                        const char *src = (const char *)a.gptr[(size_t)(r0 + r) * a.T + sg.tensor] + ((size_t)sg.off + c0) * E;
-                        bulk_load(stage_mem + (size_t)st * stage_bytes + (size_t)r * kRowBytes, src, (unsigned)tc * E,
-                                  &full_bar[st], policy);
+                        const char *src = (const char *)a.gptr[(size_t)(r0 + r) * T + k] + (size_t)c0 * E;
+                        bulk_load(dst + (size_t)r * kRowBytes, src, (unsigned)tc * E, &full_bar[st], policy);
                     }
                 }
             }
@@ -658,82 +493,88 @@ __global__ void __launch_bounds__(kStagedThreads, 2) k_reduce_staged(const __gri
         }
     } else {
         float c[CPT], s1[CPT], s2[CPT], p1[CPT], x[CPT];
-        for (int sidx = a.first[blockIdx.x]; sidx < seg_end && !timed_out; ++sidx) {
-            const Segment sg = a.segs[sidx];
-            float *gb = a.gbar + sg.goff;
-            int first_scalar = 0;
-            if (a.gflags[sg.tensor] & 1u) {
-                const int cols = sg.len & ~7;
-                first_scalar = cols;
-                for (int c0 = 0; c0 < cols && !timed_out; c0 += kTile) {
-                    const int tc = cols - c0 < kTile ? cols - c0 : kTile;
-                    const bool active = tid * CPT < tc;
-                    for (int ch = 0; ch < n_chunks; ++ch, ++item) {
-                        const int st = item % kStages;
-                        const unsigned use = item / kStages;
-                        if (!mbar_wait(&full_bar[st], use & 1u)) { timed_out = true; break; }
-                        const int r0 = ch * rps;
-                        const int rows = S - r0 < rps ? S - r0 : rps;
-                        const char *base = (const char *)stage_mem + (size_t)st * stage_bytes + (size_t)tid * CPT * E;
-                        if (active) {
-                            if (ch == 0) {
-                                if (S >= 3) {  // shift = median of the first three rows
-                                    float x1[CPT], x2[CPT];
-                                    Cols<DT, CPT>::load(base, x);
-                                    Cols<DT, CPT>::load(base + kRowBytes, x1);
-                                    Cols<DT, CPT>::load(base + 2 * kRowBytes, x2);
+        for (long long t = blockIdx.x; t < n_tiles && !timed_out; t += gridDim.x) {
+            while (t >= a.tprefix[k + 1]) ++k;
+            const long long c0 = (t - a.tprefix[k]) * kTile;
+            const long long cols = a.numel[k] & ~7LL;
+            const int tc = cols - c0 < kTile ? (int)(cols - c0) : kTile;
+            const bool active = tid * CPT < tc;
+            for (int ch = 0; ch < n_chunks; ++ch, ++item) {
+                const int st = item % kStages;
+                const unsigned use = item / kStages;
+                if (!mbar_wait(&full_bar[st], use & 1u)) { timed_out = true; break; }
+                const int r0 = ch * rps;
+                const int rows = S - r0 < rps ? S - r0 : rps;
+                const char *base = (const char *)stage_mem + (size_t)st * stage_bytes + (size_t)tid * CPT * E;
+                if (active) {
+                    if (ch == 0) {
+                        if (S >= 3) {  // shift = median of the first three rows
+                            float x1[CPT], x2[CPT];
+                            Cols<DT, CPT>::load(base, x);
+                            Cols<DT, CPT>::load(base + kRowBytes, x1);
+                            Cols<DT, CPT>::load(base + 2 * kRowBytes, x2);
 #pragma unroll
-                                    for (int k = 0; k < CPT; ++k) {
-                                        const float lo = fminf(x[k], x1[k]), hi = fmaxf(x[k], x1[k]);
-                                        c[k] = fmaxf(lo, fminf(hi, x2[k]));
-                                    }
-                                } else {
-                                    Cols<DT, CPT>::load(base, c);
-                                }
-#pragma unroll
-                                for (int k = 0; k < CPT; ++k) s1[k] = s2[k] = 0.f;
+                            for (int j = 0; j < CPT; ++j) {
+                                const float lo = fminf(x[j], x1[j]), hi = fmaxf(x[j], x1[j]);
+                                c[j] = fmaxf(lo, fminf(hi, x2[j]));
                             }
-                            for (int r = 0; r < rows; r += 8) {  // s1 in blocks of 8 rows
+                        } else {
+                            Cols<DT, CPT>::load(base, c);
+                        }
 #pragma unroll
-                                for (int k = 0; k < CPT; ++k) p1[k] = 0.f;
+                        for (int j = 0; j < CPT; ++j) s1[j] = s2[j] = 0.f;
+                    }
+                    for (int r = 0; r < rows; r += 8) {
 #pragma unroll
-                                for (int rr = 0; rr < 8; ++rr) {
-                                    if (r + rr < rows) {
-                                        Cols<DT, CPT>::load(base + (size_t)(r + rr) * kRowBytes, x);
-                                        accumulate_row<CPT>(x, c, p1, s2);
-                                    }
-                                }
+                        for (int j = 0; j < CPT; ++j) p1[j] = 0.f;
 #pragma unroll
-                                for (int k = 0; k < CPT; ++k) s1[k] += p1[k];
+                        for (int rr = 0; rr < 8; ++rr) {
+                            if (r + rr < rows) {
+                                Cols<DT, CPT>::load(base + (size_t)(r + rr) * kRowBytes, x);
+                                accumulate_row<CPT>(x, c, p1, s2);
                             }
                         }
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&empty_bar[st]);  // this warp is done with the stage
-                        if (active && ch == n_chunks - 1) {
-                            float m[CPT];
-                            float dacc = 0.f, nacc = 0.f;
 #pragma unroll
-                            for (int k = 0; k < CPT; ++k) {
-                                float qk = s1[k] * a.invS;
-                                const float res = fmaf(-qk, a.fS, s1[k]);
-                                qk = fmaf(res, a.invS, qk);
-                                m[k] = c[k] + qk;
-                                dacc += fmaf(-qk, s1[k], s2[k]);
-                                nacc = fmaf(m[k], m[k], nacc);
-                            }
-                            store_cols<CPT>(gb + c0 + tid * CPT, m);
-                            accD += (double)dacc;
-                            accN += (double)nacc;
-                        }
+                        for (int j = 0; j < CPT; ++j) s1[j] += p1[j];
                     }
                 }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty_bar[st]);  // this warp is done with the stage
+                if (active && ch == n_chunks - 1) {
+                    float m[CPT];
+                    float dacc = 0.f, nacc = 0.f;
+#pragma unroll
+                    for (int j = 0; j < CPT; ++j) {
+                        // quotient s1/S: reciprocal multiply plus one residual correction (1/S is not
+                        // exact unless S is a power of two, and a biased 1/S would bias every column alike)
+                        float q = s1[j] * a.invS;
+                        const float res = fmaf(-q, a.fS, s1[j]);
+                        q = fmaf(res, a.invS, q);
+                        m[j] = c[j] + q;
+                        dacc += fmaf(-q, s1[j], s2[j]);
+                        nacc = fmaf(m[j], m[j], nacc);
+                    }
+                    store_cols<CPT>(a.gbar + a.goff[k] + c0 + tid * CPT, m);
+                    accD += (double)dacc;
+                    accN += (double)nacc;
+                }
             }
-            // ragged tail (< 8 elements) or a tensor that is not 16-byte aligned: plain loads
-            for (int e = first_scalar + tid; e < sg.len && !timed_out; e += kConsumers) {
-                float d, n;
-                column_scalar_direct<DT>(a.gptr, a.T, sg.tensor, ((size_t)sg.off + e) * E, S, a.fS, gb + e, d, n);
+        }
+        // ragged tails (< 8 elements) and tensors that are not 16-byte aligned: plain loads
+        const long long n_stiles = a.sprefix[T];
+        int k2 = 0;
+        for (long long t = blockIdx.x; t < n_stiles; t += gridDim.x) {
+            while (t >= a.sprefix[k2 + 1]) ++k2;
+            const long long n = a.numel[k2];
+            const long long start = (a.gflags[k2] & 1u) ? (n & ~7LL) : 0;
+            const long long first = start + (t - a.sprefix[k2]) * kScalarTile;
+            const int len = n - first < kScalarTile ? (int)(n - first) : kScalarTile;
+            float *gb = a.gbar + a.goff[k2] + first;
+            for (int e = tid; e < len; e += kThreads) {
+                float d, nn;
+                column_scalar<DT>(a.gptr, T, k2, ((size_t)first + e) * E, S, a.fS, gb + e, d, nn);
                 accD += (double)d;
-                accN += (double)n;
+                accN += (double)nn;
             }
         }
         if (timed_out) atomicExch(&abort_flag, 1);
@@ -750,6 +591,8 @@ __global__ void __launch_bounds__(kStagedThreads, 2) k_reduce_staged(const __gri
     __syncthreads();
     if (!is_last) return;
 
+    // Second stage, fixed order: thread j adds partials j, j+288, ... in index order, then the
+    // same block tree.  The result depends on the tiling only, not on how blocks were scheduled.
     __threadfence();
     double d = 0.0, n = 0.0;
     for (int i = tid; i < (int)gridDim.x; i += kStagedThreads) {
@@ -764,41 +607,73 @@ __global__ void __launch_bounds__(kStagedThreads, 2) k_reduce_staged(const __gri
     }
 }
 
+// ---------------------------------------------------------------------------------------
+// Update kernel (Eq. 2 with momentum): tiles of kUpdateTile elements, one 128-bit access per
+// array and thread, tiles dealt round-robin like in the reduce kernel.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void update4(float4 &ww, float4 &vv, const float4 &gg, float rho, float lambda, float eta)
+{
+    vv.x = fmaf(rho, vv.x, fmaf(lambda, ww.x, gg.x));
+    vv.y = fmaf(rho, vv.y, fmaf(lambda, ww.y, gg.y));
+    vv.z = fmaf(rho, vv.z, fmaf(lambda, ww.z, gg.z));
+    vv.w = fmaf(rho, vv.w, fmaf(lambda, ww.w, gg.w));
+    ww.x = fmaf(-eta, vv.x, ww.x);
+    ww.y = fmaf(-eta, vv.y, ww.y);
+    ww.z = fmaf(-eta, vv.z, ww.z);
+    ww.w = fmaf(-eta, vv.w, ww.w);
+}
+
 __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const __grid_constant__ UpdateArgs a)
 {
     if (a.st->status & ADASCALE_STATUS_NONFINITE) return;
     const float eta = (float)a.st->eta;
-    const int tid = threadIdx.x;
-    const int seg_end = a.first[blockIdx.x + 1];
-    for (int sidx = a.first[blockIdx.x]; sidx < seg_end; ++sidx) {
-        const Segment sg = a.segs[sidx];
-        float *w = (float *)a.wv[sg.tensor] + sg.off;
-        float *v = (float *)a.wv[a.T + sg.tensor] + sg.off;
-        const float *g = a.gbar + sg.goff;
-        int first_scalar = 0;
-        if (a.wflags[sg.tensor] & 1u) {
-            const int nv = sg.len >> 2;
-            for (int i = tid; i < nv; i += kThreads) {
-                const float4 gg = ((const float4 *)g)[i];
-                float4 ww = ((const float4 *)w)[i];
-                float4 vv = ((const float4 *)v)[i];
-                vv.x = fmaf(a.rho, vv.x, fmaf(a.lambda, ww.x, gg.x));
-                vv.y = fmaf(a.rho, vv.y, fmaf(a.lambda, ww.y, gg.y));
-                vv.z = fmaf(a.rho, vv.z, fmaf(a.lambda, ww.z, gg.z));
-                vv.w = fmaf(a.rho, vv.w, fmaf(a.lambda, ww.w, gg.w));
-                ww.x = fmaf(-eta, vv.x, ww.x);
-                ww.y = fmaf(-eta, vv.y, ww.y);
-                ww.z = fmaf(-eta, vv.z, ww.z);
-                ww.w = fmaf(-eta, vv.w, ww.w);
-                ((float4 *)v)[i] = vv;
-                ((float4 *)w)[i] = ww;
-            }
-            first_scalar = nv << 2;
+    const int tid = threadIdx.x, T = a.T;
+    const long long n_tiles = a.uprefix[T];
+    int k = 0, held = -1;
+    float *wp = nullptr, *vp = nullptr;
+    const float *gp = nullptr;
+    long long n = 0;
+    bool vec = false;
+    for (long long t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+        while (t >= a.uprefix[k + 1]) ++k;
+        if (k != held) {  // tiles only move forward, so a tensor's pointers are fetched once
+            held = k;
+            wp = (float *)a.wv[k];
+            vp = (float *)a.wv[T + k];
+            gp = a.gbar + a.goff[k];
+            n = a.numel[k];
+            vec = (a.wflags[k] & 1u) != 0;
         }
-        for (int e = first_scalar + tid; e < sg.len; e += kThreads) {
-            const float vn = fmaf(a.rho, v[e], fmaf(a.lambda, w[e], g[e]));
-            v[e] = vn;
-            w[e] = fmaf(-eta, vn, w[e]);
+        const long long first = (t - a.uprefix[k]) * kUpdateTile;
+        const int len = n - first < kUpdateTile ? (int)(n - first) : kUpdateTile;
+        float *w = wp + first, *v = vp + first;
+        const float *g = gp + first;
+        if (vec && len == kUpdateTile) {
+            const float4 gg = ((const float4 *)g)[tid];
+            float4 ww = ((const float4 *)w)[tid];
+            float4 vv = ((const float4 *)v)[tid];
+            update4(ww, vv, gg, a.rho, a.lambda, eta);
+            ((float4 *)v)[tid] = vv;
+            ((float4 *)w)[tid] = ww;
+        } else {
+            int done = 0;
+            if (vec) {
+                const int nv = len >> 2;
+                if (tid < nv) {
+                    const float4 gg = ((const float4 *)g)[tid];
+                    float4 ww = ((const float4 *)w)[tid];
+                    float4 vv = ((const float4 *)v)[tid];
+                    update4(ww, vv, gg, a.rho, a.lambda, eta);
+                    ((float4 *)v)[tid] = vv;
+                    ((float4 *)w)[tid] = ww;
+                }
+                done = nv << 2;
+            }
+            for (int e = done + tid; e < len; e += kThreads) {
+                const float vn = fmaf(a.rho, v[e], fmaf(a.lambda, w[e], g[e]));
+                v[e] = vn;
+                w[e] = fmaf(-eta, vn, w[e]);
+            }
         }
     }
 }
@@ -835,11 +710,11 @@ __global__ void __launch_bounds__(kThreads) k_probe_rmw(float4 *a, const float4 
 // host side
 // ---------------------------------------------------------------------------------------
 
-// A table of pointers (plus per-tensor flags) mirrored on the host and uploaded only when
-// it changes, through a small ring of pinned slots so that an upload still in flight is
-// never overwritten.
+// A table of pointers (plus per-tensor flags and tile prefixes) mirrored on the host and
+// uploaded only when it changes, through a small ring of pinned slots so that an upload
+// still in flight is never overwritten.
 struct PtrTable {
-    std::vector<u64> mirror;   // last uploaded contents (pointers then flags, 8-byte units)
+    std::vector<u64> mirror;   // last uploaded contents, 8-byte words
     u64 *dev = nullptr;
     u64 *pinned[kRing] = {nullptr, nullptr, nullptr, nullptr};
     cudaEvent_t ev[kRing] = {nullptr, nullptr, nullptr, nullptr};
@@ -864,31 +739,31 @@ constexpr unsigned kMagic = 0x41645363u;  // "AdSc"
 }  // namespace
 
 struct adascale_ctx {
-    int device = 0;
+    int device = 0, sms = 0;
     int S = 1, max_S = 1, T = 0, dtype = 0;
     double rho = 0, lambda = 0, eps = 1e-6, theta_cfg = -1;
     unsigned flags = 0;
     std::vector<long long> numel;
     std::vector<long long> goff;
+    std::vector<long long> uprefix;
     long long P = 0, gbar_elems = 0;
-    Plan plan_r, plan_u;          // reduce and update kernels
-    bool staged = true;
-    Segment *d_segs_r = nullptr, *d_segs_u = nullptr;
-    int *d_first_r = nullptr, *d_first_u = nullptr;
+    long long *d_numel = nullptr, *d_goff = nullptr, *d_uprefix = nullptr;
     float *d_gbar = nullptr;
     double2 *d_partials = nullptr;
     unsigned *d_ticket = nullptr;
     DevState *d_state = nullptr;
     PtrTable tg, tw;
-    DevState *h_snap = nullptr;      // pinned, 2 slots
+    // tiling of the last reduce table
+    int cpt = 0;
+    long long n_tiles = 0, n_stiles = 0;
+    DevState *h_snap = nullptr;  // pinned
     cudaEvent_t ev_snap = nullptr;
     bool snap_inflight = false;
     DevState latest{};
     cudaStream_t last_stream = nullptr;
     bool reduced = false;
     long long launches = 0;
-    // host-gradient staging (adascale_step_host)
-    void *d_stage = nullptr;
+    void *d_stage = nullptr;     // host-gradient staging (adascale_step_host)
     std::vector<const void *> stage_ptrs;
     std::string err;
 };
@@ -927,76 +802,57 @@ adascale_status cuda_fail(adascale_ctx *c, cudaError_t e, const char *what)
         if (e_ != cudaSuccess) return cuda_fail(ctx, e_, #call);    \
     } while (0)
 
-// Splits the tensors over at most max_blocks blocks so that every block gets the same cost,
-// where a segment costs its length in units (one unit = `unit` elements, the width of a
-// vector access) plus a fixed `seg_cost` for staging its row pointers.  Segment boundaries
-// are multiples of `unit` elements from the tensor's start, so a 16-byte aligned tensor
-// stays 16-byte aligned in every segment.
-Plan make_plan(const std::vector<long long> &numel, const std::vector<long long> &goff, int unit,
-               long long seg_cost, int max_blocks)
-{
-    Plan p;
-    long long units_total = 0, tensors = 0;
-    for (long long n : numel)
-        if (n > 0) {
-            units_total += (n + unit - 1) / unit;
-            tensors += 1;
-        }
-    if (units_total == 0) {
-        p.n_blocks = 0;
-        p.first.assign(1, 0);
-        return p;
-    }
-    long long nb = (units_total + kMinUnitsPerBlock - 1) / kMinUnitsPerBlock;
-    if (nb > max_blocks) nb = max_blocks;
-    if (nb < 1) nb = 1;
-    // every block boundary that falls inside a tensor adds one more segment
-    const long long cost_total = units_total + seg_cost * (tensors + nb - 1);
-    const long long target = (cost_total + nb - 1) / nb;
-    p.n_blocks = (int)nb;
-    p.first.assign((size_t)nb + 1, 0);
-    long long b = 0, acc = 0;
-    for (size_t k = 0; k < numel.size(); ++k) {
-        const long long n = numel[k];
-        long long rem = n > 0 ? (n + unit - 1) / unit : 0, off = 0;
-        while (rem > 0) {
-            if (b < nb - 1 && acc > 0 && acc + seg_cost + 1 > target) {  // not worth starting here
-                p.first[(size_t)++b] = (int)p.segs.size();
-                acc = 0;
-            }
-            long long room = target - acc - seg_cost;
-            if (room < 1) room = 1;
-            const long long take = (b == nb - 1 || rem < room) ? rem : room;
-            Segment sg;
-            sg.tensor = (int)k;
-            sg.off = off * unit;
-            sg.goff = goff[k] + sg.off;
-            const long long len = (sg.off + take * unit <= n) ? take * unit : n - sg.off;
-            sg.len = (int)len;
-            p.segs.push_back(sg);
-            acc += take + seg_cost;
-            off += take;
-            rem -= take;
-        }
-    }
-    while (b < nb) p.first[(size_t)++b] = (int)p.segs.size();
-    return p;
-}
-
-// Fixed cost of one segment in units: staging S row pointers takes about as long as
-// streaming ~16 KB does at one block's share of the bandwidth, and a unit is 16*S bytes.
-long long segment_cost(int S)
-{
-    const long long c = 1024 / (S > 0 ? S : 1);
-    return c < 4 ? 4 : c;
-}
-
 double resolve_theta(const adascale_ctx *c)
 {
     if (c->theta_cfg >= 0.0) return c->theta_cfg;
     const double th = 1.0 - (double)c->S / 1000.0;  // Sec. 3.4: theta = max{1 - S/1000, 0}
     return th > 0.0 ? th : 0.0;
 }
+
+// ---- tiling of the reduce kernel ---------------------------------------------------------
+
+int rows_per_stage(int S) { return S < kMaxRowsPerStage ? S : kMaxRowsPerStage; }
+
+long long staged_tiles(const long long *numel, const unsigned char *aligned, int T, int tile_cols)
+{
+    long long n = 0;
+    for (int k = 0; k < T; ++k)
+        if (!aligned || aligned[k]) n += ((numel[k] & ~7LL) + tile_cols - 1) / tile_cols;
+    return n;
+}
+
+// Columns per consumer thread.  A thread reads 8, 16 or 32 bytes of each row; the widest
+// access that keeps one stage (rows x 256 threads x bytes) within kStageBytes is used, and
+// small jobs step down so that every block still gets a few tiles.
+int choose_cpt(int dtype, int S, const long long *numel, const unsigned char *aligned, int T, int n_blocks)
+{
+    const int esz = dtype == ADASCALE_BF16 ? 2 : 4;
+    int bpt = dtype == ADASCALE_BF16 ? 16 : 32;
+    while (bpt > 8 && rows_per_stage(S) * kThreads * bpt > kStageBytes) bpt >>= 1;
+    while (bpt > 8 && staged_tiles(numel, aligned, T, kThreads * bpt / esz) < 4LL * n_blocks) bpt >>= 1;
+    return bpt / esz;
+}
+
+void build_prefixes(const long long *numel, const unsigned char *aligned, int T, int tile_cols,
+                    long long *tprefix, long long *sprefix)
+{
+    long long nt = 0, ns = 0;
+    for (int k = 0; k < T; ++k) {
+        tprefix[k] = nt;
+        sprefix[k] = ns;
+        const long long n = numel[k];
+        if (!aligned || aligned[k]) {
+            nt += ((n & ~7LL) + tile_cols - 1) / tile_cols;
+            ns += (n & 7LL) ? 1 : 0;
+        } else {
+            ns += (n + kScalarTile - 1) / kScalarTile;
+        }
+    }
+    tprefix[T] = nt;
+    sprefix[T] = ns;
+}
+
+// ---- pointer tables ----------------------------------------------------------------------
 
 adascale_status table_alloc(adascale_ctx *ctx, PtrTable &t, size_t words)
 {
@@ -1042,68 +898,33 @@ adascale_status table_sync(adascale_ctx *ctx, PtrTable &t, const std::vector<u64
     return ADASCALE_OK;
 }
 
-template <int DT>
-cudaError_t launch_reduce(int B, int n_blocks, const ReduceArgs &a, size_t smem, cudaStream_t s)
-{
-    const dim3 grid(n_blocks), block(kThreads);
-    switch (B) {
-    case 1: k_reduce<DT, 1><<<grid, block, smem, s>>>(a); break;
-    case 2: k_reduce<DT, 2><<<grid, block, smem, s>>>(a); break;
-    case 4: k_reduce<DT, 4><<<grid, block, smem, s>>>(a); break;
-    default: k_reduce<DT, 8><<<grid, block, smem, s>>>(a); break;
-    }
-    return cudaGetLastError();
-}
-
-int batch_for(int S) { return S >= 8 ? 8 : S >= 4 ? 4 : S >= 2 ? 2 : 1; }
-
-// Columns per consumer thread: as many as keep one stage (rows x 256 x CPT elements) within 32 KB.
-int cols_per_thread(int dtype, int S)
-{
-    const int rps = S < kRowsPerStage ? S : kRowsPerStage;
-    const int budget = (dtype == ADASCALE_BF16 ? 64 : 32) / rps;
-    int cpt = 8;
-    while (cpt > budget && cpt > 1) cpt >>= 1;
-    if (dtype == ADASCALE_BF16 && cpt < 2) cpt = 2;
-    return cpt;
-}
-
-size_t staged_smem(int dtype, int S, int cpt)
-{
-    const int rps = S < kRowsPerStage ? S : kRowsPerStage;
-    return (size_t)kStages * rps * kConsumers * cpt * (dtype == ADASCALE_BF16 ? 2 : 4);
-}
+// ---- launches ----------------------------------------------------------------------------
 
 template <int DT, int CPT>
-cudaError_t launch_staged_one(int n_blocks, const ReduceArgs &a, size_t smem, cudaStream_t s)
+cudaError_t launch_reduce_one(int n_blocks, const ReduceArgs &a, size_t smem, cudaStream_t s)
 {
     static bool configured[64] = {false};
     int dev = 0;
     cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(k_reduce_staged<DT, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)(kStages * 32 * 1024));
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(k_reduce<DT, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kStages * kStageBytes);
         if (e != cudaSuccess) return e;
-        configured[dev] = true;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    k_reduce_staged<DT, CPT><<<dim3(n_blocks), dim3(kStagedThreads), smem, s>>>(a);
+    k_reduce<DT, CPT><<<dim3(n_blocks), dim3(kStagedThreads), smem, s>>>(a);
     return cudaGetLastError();
 }
 
-cudaError_t launch_staged(int dtype, int cpt, int n_blocks, const ReduceArgs &a, size_t smem, cudaStream_t s)
+cudaError_t launch_reduce(int dtype, int cpt, int n_blocks, const ReduceArgs &a, size_t smem, cudaStream_t s)
 {
-    if (dtype == ADASCALE_BF16) {
-        switch (cpt) {
-        case 2: return launch_staged_one<ADASCALE_BF16, 2>(n_blocks, a, smem, s);
-        case 4: return launch_staged_one<ADASCALE_BF16, 4>(n_blocks, a, smem, s);
-        default: return launch_staged_one<ADASCALE_BF16, 8>(n_blocks, a, smem, s);
-        }
-    }
+    if (dtype == ADASCALE_BF16)
+        return cpt == 4 ? launch_reduce_one<ADASCALE_BF16, 4>(n_blocks, a, smem, s)
+                        : launch_reduce_one<ADASCALE_BF16, 8>(n_blocks, a, smem, s);
     switch (cpt) {
-    case 1: return launch_staged_one<ADASCALE_F32, 1>(n_blocks, a, smem, s);
-    case 2: return launch_staged_one<ADASCALE_F32, 2>(n_blocks, a, smem, s);
-    case 4: return launch_staged_one<ADASCALE_F32, 4>(n_blocks, a, smem, s);
-    default: return launch_staged_one<ADASCALE_F32, 8>(n_blocks, a, smem, s);
+    case 2: return launch_reduce_one<ADASCALE_F32, 2>(n_blocks, a, smem, s);
+    case 4: return launch_reduce_one<ADASCALE_F32, 4>(n_blocks, a, smem, s);
+    default: return launch_reduce_one<ADASCALE_F32, 8>(n_blocks, a, smem, s);
     }
 }
 
@@ -1118,35 +939,46 @@ bool valid_sched(const adascale_lr_schedule *s)
     return true;
 }
 
+// Layout of the reduce table in 8-byte words:
+//   [max_S * T row pointers][T + 1 staged-tile prefix][T + 1 scalar-tile prefix][ceil(T/2) flags]
 adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const adascale_lr_schedule *sched,
                           cudaStream_t s)
 {
     const int S = ctx->S, T = ctx->T;
     const size_t esz = ctx->dtype == ADASCALE_BF16 ? 2 : 4;
+    const size_t w_ptr = 0, w_tp = (size_t)ctx->max_S * T, w_sp = w_tp + T + 1, w_fl = w_sp + T + 1;
     std::vector<u64> fresh(ctx->tg.words, 0);
-    unsigned *flags = reinterpret_cast<unsigned *>(fresh.data() + (size_t)ctx->max_S * T);
+    std::vector<unsigned char> aligned((size_t)T, 1);
+    unsigned *flags = reinterpret_cast<unsigned *>(fresh.data() + w_fl);
     for (int k = 0; k < T; ++k) {
-        unsigned aligned = 1u;
         for (int i = 0; i < S; ++i) {
             const u64 p = (u64)(uintptr_t)grads[(size_t)i * T + k];
             if (ctx->numel[k] > 0) {
                 if (p == 0) return ADASCALE_ERR_INVALID_ARG;
                 if (p % esz) return ADASCALE_ERR_ALIGNMENT;
-                if (p % 16) aligned = 0u;
+                if (p % 16) aligned[k] = 0;
             }
-            fresh[(size_t)i * T + k] = p;
+            fresh[w_ptr + (size_t)i * T + k] = p;
         }
-        flags[k] = aligned;
+        flags[k] = aligned[k];
     }
+    const int max_blocks = ctx->sms * kReduceBlocksPerSM;
+    const int cpt = choose_cpt(ctx->dtype, S, ctx->numel.data(), aligned.data(), T, max_blocks);
+    build_prefixes(ctx->numel.data(), aligned.data(), T, kThreads * cpt,
+                   reinterpret_cast<long long *>(fresh.data() + w_tp),
+                   reinterpret_cast<long long *>(fresh.data() + w_sp));
+    const long long n_tiles = (long long)fresh[w_tp + T], n_stiles = (long long)fresh[w_sp + T];
     adascale_status st = table_sync(ctx, ctx->tg, fresh, s);
     if (st != ADASCALE_OK) return st;
-    if (ctx->plan_r.n_blocks == 0) return ADASCALE_OK;
+    if (n_tiles + n_stiles == 0) return ADASCALE_OK;  // nothing but empty tensors
 
     ReduceArgs a;
-    a.segs = ctx->d_segs_r;
-    a.first = ctx->d_first_r;
-    a.gptr = ctx->tg.dev;
-    a.gflags = reinterpret_cast<const unsigned *>(ctx->tg.dev + (size_t)ctx->max_S * T);
+    a.gptr = ctx->tg.dev + w_ptr;
+    a.tprefix = reinterpret_cast<const long long *>(ctx->tg.dev + w_tp);
+    a.sprefix = reinterpret_cast<const long long *>(ctx->tg.dev + w_sp);
+    a.gflags = reinterpret_cast<const unsigned *>(ctx->tg.dev + w_fl);
+    a.numel = ctx->d_numel;
+    a.goff = ctx->d_goff;
     a.gbar = ctx->d_gbar;
     a.partials = ctx->d_partials;
     a.ticket = ctx->d_ticket;
@@ -1166,24 +998,21 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
     a.sched.t_s1 = sched->t_s1;
     for (int i = 0; i < ADASCALE_MAX_MILESTONES; ++i) a.sched.w[i] = sched->milestones[i];
 
-    const size_t smem = (size_t)S * sizeof(u64);
-    const int B = batch_for(S);
-    const int nb = ctx->plan_r.n_blocks;
-    cudaError_t e;
-    if (ctx->staged) {
-        const int cpt = cols_per_thread(ctx->dtype, S);
-        e = launch_staged(ctx->dtype, cpt, nb, a, staged_smem(ctx->dtype, S, cpt), s);
-    } else {
-        e = ctx->dtype == ADASCALE_BF16 ? launch_reduce<ADASCALE_BF16>(B, nb, a, smem, s)
-                                        : launch_reduce<ADASCALE_F32>(B, nb, a, smem, s);
-    }
+    long long nb = n_tiles + n_stiles;
+    if (nb > max_blocks) nb = max_blocks;
+    const size_t smem = (size_t)kStages * rows_per_stage(S) * kThreads * cpt * esz;
+    cudaError_t e = launch_reduce(ctx->dtype, cpt, (int)nb, a, smem, s);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "launch of the reduce kernel");
+    ctx->cpt = cpt;
+    ctx->n_tiles = n_tiles;
+    ctx->n_stiles = n_stiles;
     ctx->launches += 1;
     ctx->reduced = true;
     ctx->last_stream = s;
     return ADASCALE_OK;
 }
 
+// Layout of the update table in 8-byte words: [T parameters][T momentum][ceil(T/2) flags]
 adascale_status do_update(adascale_ctx *ctx, void *const *params, void *const *momentum, cudaStream_t s)
 {
     const int T = ctx->T;
@@ -1201,19 +1030,23 @@ adascale_status do_update(adascale_ctx *ctx, void *const *params, void *const *m
     }
     adascale_status st = table_sync(ctx, ctx->tw, fresh, s);
     if (st != ADASCALE_OK) return st;
-    if (ctx->plan_u.n_blocks == 0) return ADASCALE_OK;
+    const long long n_tiles = ctx->uprefix[(size_t)T];
+    if (n_tiles == 0) return ADASCALE_OK;
 
     UpdateArgs a;
-    a.segs = ctx->d_segs_u;
-    a.first = ctx->d_first_u;
     a.wv = ctx->tw.dev;
     a.wflags = reinterpret_cast<const unsigned *>(ctx->tw.dev + (size_t)2 * T);
+    a.uprefix = ctx->d_uprefix;
+    a.numel = ctx->d_numel;
+    a.goff = ctx->d_goff;
     a.gbar = ctx->d_gbar;
     a.st = ctx->d_state;
     a.T = T;
     a.rho = (float)ctx->rho;
     a.lambda = (float)ctx->lambda;
-    k_update<<<dim3(ctx->plan_u.n_blocks), dim3(kThreads), 0, s>>>(a);
+    long long nb = n_tiles;
+    if (nb > (long long)ctx->sms * kUpdateBlocksPerSM) nb = (long long)ctx->sms * kUpdateBlocksPerSM;
+    k_update<<<dim3((unsigned)nb), dim3(kThreads), 0, s>>>(a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(ctx, e, "launch of the update kernel");
     ctx->launches += 1;
@@ -1221,7 +1054,7 @@ adascale_status do_update(adascale_ctx *ctx, void *const *params, void *const *m
     return ADASCALE_OK;
 }
 
-void fill_stats(const adascale_ctx *ctx, const DevState &d, adascale_stats *o)
+void fill_stats(const DevState &d, adascale_stats *o)
 {
     std::memset(o, 0, sizeof *o);
     o->r = d.r;
@@ -1238,7 +1071,6 @@ void fill_stats(const adascale_ctx *ctx, const DevState &d, adascale_stats *o)
     o->n_samples = d.n;
     o->skipped = d.skipped;
     o->status_bits = d.status | d.fault;
-    (void)ctx;
 }
 
 }  // namespace
@@ -1262,29 +1094,26 @@ const char *adascale_last_error(const adascale_ctx *ctx) { return ctx ? ctx->err
 
 int64_t adascale_launch_count(const adascale_ctx *ctx) { return ctx ? ctx->launches : 0; }
 
-int64_t adascale_plan(const int64_t *numel, int32_t n_tensors, int32_t unit, int64_t seg_cost,
-                      int32_t max_blocks, int64_t *out, int64_t cap)
+adascale_status adascale_tiling(const int64_t *numel, int32_t n_tensors, int32_t grad_dtype, int32_t S,
+                                const uint8_t *aligned, int32_t n_blocks, int64_t *tprefix, int64_t *sprefix,
+                                int32_t *tile_cols, int32_t *rows)
 {
-    if (!numel || n_tensors < 1 || unit < 1 || seg_cost < 0 || max_blocks < 1 || cap < 0 || (cap > 0 && !out))
-        return -1;
-    std::vector<long long> n(numel, numel + n_tensors), goff;
-    long long g = 0;
-    for (long long x : n) {
-        if (x < 0) return -1;
-        goff.push_back(g);
-        g += (x + kGbarAlign - 1) / kGbarAlign * kGbarAlign;
+    if (!numel || n_tensors < 1 || S < 1 || n_blocks < 1 || !tprefix || !sprefix || !tile_cols || !rows)
+        return ADASCALE_ERR_INVALID_ARG;
+    if (grad_dtype != ADASCALE_F32 && grad_dtype != ADASCALE_BF16) return ADASCALE_ERR_INVALID_ARG;
+    std::vector<long long> n(numel, numel + n_tensors);
+    for (long long x : n)
+        if (x < 0) return ADASCALE_ERR_INVALID_ARG;
+    const int cpt = choose_cpt(grad_dtype, S, n.data(), aligned, n_tensors, n_blocks);
+    std::vector<long long> tp((size_t)n_tensors + 1), sp((size_t)n_tensors + 1);
+    build_prefixes(n.data(), aligned, n_tensors, kThreads * cpt, tp.data(), sp.data());
+    for (int k = 0; k <= n_tensors; ++k) {
+        tprefix[k] = tp[(size_t)k];
+        sprefix[k] = sp[(size_t)k];
     }
-    const Plan p = make_plan(n, goff, unit, seg_cost, max_blocks);
-    int64_t written = 0;
-    for (int b = 0; b < p.n_blocks; ++b)
-        for (int i = p.first[b]; i < p.first[b + 1]; ++i, ++written)
-            if (written < cap) {
-                out[4 * written + 0] = p.segs[i].tensor;
-                out[4 * written + 1] = p.segs[i].off;
-                out[4 * written + 2] = p.segs[i].len;
-                out[4 * written + 3] = b;
-            }
-    return (int64_t)p.segs.size();
+    *tile_cols = kThreads * cpt;
+    *rows = rows_per_stage(S);
+    return ADASCALE_OK;
 }
 
 adascale_status adascale_init(const adascale_config *cfg, adascale_ctx **out)
@@ -1317,50 +1146,37 @@ adascale_status adascale_init(const adascale_config *cfg, adascale_ctx **out)
     ctx->flags = cfg->flags;
     ctx->numel.assign(cfg->numel, cfg->numel + cfg->n_tensors);
 
-    long long g = 0;
+    long long g = 0, ut = 0;
     for (int k = 0; k < ctx->T; ++k) {
-        ctx->goff.push_back(g);
         const long long n = ctx->numel[k];
+        ctx->goff.push_back(g);
+        ctx->uprefix.push_back(ut);
         ctx->P += n;
         g += (n + kGbarAlign - 1) / kGbarAlign * kGbarAlign;
+        ut += (n + kUpdateTile - 1) / kUpdateTile;
     }
+    ctx->uprefix.push_back(ut);
     ctx->gbar_elems = g;
 
     DeviceGuard guard(ctx->device);
-    adascale_status rc = ADASCALE_OK;
     auto body = [&]() -> adascale_status {
         if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
-        int sms = 0;
-        CU(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device));
-        // one plan per kernel: the grid is sized to the device, the split is fixed from here on,
-        // which is what makes the fixed-order sums reproducible from run to run
-        ctx->staged = std::getenv("ADASCALE_REDUCE_LDG") == nullptr;
-        ctx->plan_r = make_plan(ctx->numel, ctx->goff, 8, segment_cost(ctx->S),
-                                sms * (ctx->staged ? 2 : kReduceBlocksPerSM));
-        ctx->plan_u = make_plan(ctx->numel, ctx->goff, 4, 64, sms * kUpdateBlocksPerSM);
-        if (ctx->plan_r.segs.size() > 0x7fffffffull) return ADASCALE_ERR_TOO_LARGE;
-        auto upload = [&](const Plan &pl, Segment **dsegs, int **dfirst) -> adascale_status {
-            const size_t ns = pl.segs.empty() ? 1 : pl.segs.size();
-            CU(cudaMalloc(dsegs, ns * sizeof(Segment)));
-            CU(cudaMalloc(dfirst, pl.first.size() * sizeof(int)));
-            if (!pl.segs.empty())
-                CU(cudaMemcpy(*dsegs, pl.segs.data(), pl.segs.size() * sizeof(Segment), cudaMemcpyHostToDevice));
-            CU(cudaMemcpy(*dfirst, pl.first.data(), pl.first.size() * sizeof(int), cudaMemcpyHostToDevice));
-            return ADASCALE_OK;
-        };
-        adascale_status s0 = upload(ctx->plan_r, &ctx->d_segs_r, &ctx->d_first_r);
-        if (s0 != ADASCALE_OK) return s0;
-        s0 = upload(ctx->plan_u, &ctx->d_segs_u, &ctx->d_first_u);
-        if (s0 != ADASCALE_OK) return s0;
+        CU(cudaDeviceGetAttribute(&ctx->sms, cudaDevAttrMultiProcessorCount, ctx->device));
+        const size_t T = (size_t)ctx->T;
+        CU(cudaMalloc(&ctx->d_numel, T * sizeof(long long)));
+        CU(cudaMalloc(&ctx->d_goff, T * sizeof(long long)));
+        CU(cudaMalloc(&ctx->d_uprefix, (T + 1) * sizeof(long long)));
+        CU(cudaMemcpy(ctx->d_numel, ctx->numel.data(), T * sizeof(long long), cudaMemcpyHostToDevice));
+        CU(cudaMemcpy(ctx->d_goff, ctx->goff.data(), T * sizeof(long long), cudaMemcpyHostToDevice));
+        CU(cudaMemcpy(ctx->d_uprefix, ctx->uprefix.data(), (T + 1) * sizeof(long long), cudaMemcpyHostToDevice));
         CU(cudaMalloc(&ctx->d_gbar, (size_t)(g > 0 ? g : 1) * sizeof(float)));
         CU(cudaMemset(ctx->d_gbar, 0, (size_t)(g > 0 ? g : 1) * sizeof(float)));
-        CU(cudaMalloc(&ctx->d_partials, (size_t)(ctx->plan_r.n_blocks + 1) * sizeof(double2)));
+        CU(cudaMalloc(&ctx->d_partials, (size_t)(ctx->sms * kReduceBlocksPerSM + 1) * sizeof(double2)));
         CU(cudaMalloc(&ctx->d_ticket, sizeof(unsigned)));
         CU(cudaMemset(ctx->d_ticket, 0, sizeof(unsigned)));
         CU(cudaMalloc(&ctx->d_state, sizeof(DevState)));
         CU(cudaMemset(ctx->d_state, 0, sizeof(DevState)));
-        const size_t T = (size_t)ctx->T;
-        adascale_status s1 = table_alloc(ctx, ctx->tg, (size_t)ctx->max_S * T + (T + 1) / 2);
+        adascale_status s1 = table_alloc(ctx, ctx->tg, (size_t)ctx->max_S * T + 2 * (T + 1) + (T + 1) / 2);
         if (s1 != ADASCALE_OK) return s1;
         s1 = table_alloc(ctx, ctx->tw, 2 * T + (T + 1) / 2);
         if (s1 != ADASCALE_OK) return s1;
@@ -1369,7 +1185,7 @@ adascale_status adascale_init(const adascale_config *cfg, adascale_ctx **out)
         CU(cudaEventCreateWithFlags(&ctx->ev_snap, cudaEventDisableTiming));
         return ADASCALE_OK;
     };
-    rc = body();
+    const adascale_status rc = body();
     if (rc != ADASCALE_OK) {
         adascale_destroy(ctx);
         return rc;
@@ -1384,10 +1200,9 @@ adascale_status adascale_destroy(adascale_ctx *ctx)
     DeviceGuard guard(ctx->device);
     if (guard.ok) {
         cudaDeviceSynchronize();
-        cudaFree(ctx->d_segs_r);
-        cudaFree(ctx->d_segs_u);
-        cudaFree(ctx->d_first_r);
-        cudaFree(ctx->d_first_u);
+        cudaFree(ctx->d_numel);
+        cudaFree(ctx->d_goff);
+        cudaFree(ctx->d_uprefix);
         cudaFree(ctx->d_gbar);
         cudaFree(ctx->d_partials);
         cudaFree(ctx->d_ticket);
@@ -1473,7 +1288,7 @@ adascale_status adascale_get_gain_tau(adascale_ctx *ctx, adascale_stats *out, in
             ctx->snap_inflight = false;
         }
     }
-    fill_stats(ctx, ctx->latest, out);
+    fill_stats(ctx->latest, out);
     return ADASCALE_OK;
 }
 
