@@ -73,17 +73,25 @@ struct Sched {
     double w[ADASCALE_MAX_MILESTONES];
 };
 
-// Tiling of the tensor list for one launch of the reduce kernel.  A tensor whose S row
-// pointers are 16-byte aligned contributes ceil(cols / tile_cols) staged tiles for its first
-// cols = numel & ~7 elements and one scalar tile for the ragged rest; any other tensor
-// contributes only scalar tiles of kScalarTile elements.
+// One tile of work: `len` elements of tensor `tensor` starting at element `first`; `goff` is
+// where the tile's mean gradient lives in the library's workspace.  Tile t belongs to block
+// t mod gridDim.  The descriptors hold no pointers, so they change only with the tiling.
+struct __align__(16) TileDesc {
+    long long first;
+    long long goff;
+    int tensor;
+    int len;
+    int pad[2];
+};
+
+// Reduce kernel: a tensor whose S row pointers are 16-byte aligned contributes staged tiles of
+// kThreads * CPT columns for its first numel & ~7 elements and one scalar tile for the ragged
+// rest; any other tensor contributes only scalar tiles of kScalarTile elements.
 struct ReduceArgs {
     const u64 *gptr;          // [S * T] row pointers
-    const long long *tprefix; // [T + 1] staged tiles before tensor k
-    const long long *sprefix; // [T + 1] scalar tiles before tensor k
-    const unsigned *gflags;   // [T] bit0: all S rows of the tensor are 16-byte aligned
-    const long long *numel;   // [T]
-    const long long *goff;    // [T] offset of the tensor in the mean-gradient workspace
+    const TileDesc *tiles;    // staged tiles
+    const TileDesc *stiles;   // scalar-path tiles
+    long long n_tiles, n_stiles;
     float *gbar;
     double2 *partials;
     unsigned *ticket;
@@ -97,19 +105,15 @@ struct ReduceArgs {
 struct UpdateArgs {
     const u64 *wv;            // [2 * T]: parameters then momentum
     const unsigned *wflags;   // [T] bit0: both pointers 16-byte aligned
-    const long long *uprefix; // [T + 1] update tiles before tensor k
-    const long long *numel;
-    const long long *goff;
+    const TileDesc *tiles;    // tiles of kUpdateTile elements
+    long long n_tiles;
     const float *gbar;
     const DevState *st;
     int T;
     float rho, lambda;
 };
 
-// ---------------------------------------------------------------------------------------
-// loads: the gradient rows are read exactly once, so they bypass L1 and are marked
-// evict-first in L2, which leaves the cache to the mean gradient the update reads next.
-// ---------------------------------------------------------------------------------------
+// Streaming 128-bit load (read once, evict first): used by the bandwidth probes.
 __device__ __forceinline__ uint4 ld_stream16(const void *p)
 {
     uint4 r;
@@ -119,32 +123,15 @@ __device__ __forceinline__ uint4 ld_stream16(const void *p)
     return r;
 }
 
+// Element types of the gradient rows.  A bf16 is the upper half of an fp32, so widening is a
+// shift and exact.
 template <int DT> struct Elem;
 template <> struct Elem<ADASCALE_F32> {
-    static constexpr int kBytes = 4, kVec = 4;
-    static __device__ __forceinline__ void unpack(const uint4 &q, float *x)
-    {
-        x[0] = __uint_as_float(q.x);
-        x[1] = __uint_as_float(q.y);
-        x[2] = __uint_as_float(q.z);
-        x[3] = __uint_as_float(q.w);
-    }
+    static constexpr int kBytes = 4;
     static __device__ __forceinline__ float load1(const void *p) { return __ldcs((const float *)p); }
 };
 template <> struct Elem<ADASCALE_BF16> {
-    static constexpr int kBytes = 2, kVec = 8;
-    // a bf16 is the upper half of an fp32: widening is a shift, exact
-    static __device__ __forceinline__ void unpack(const uint4 &q, float *x)
-    {
-        x[0] = __uint_as_float(q.x << 16);
-        x[1] = __uint_as_float(q.x & 0xffff0000u);
-        x[2] = __uint_as_float(q.y << 16);
-        x[3] = __uint_as_float(q.y & 0xffff0000u);
-        x[4] = __uint_as_float(q.z << 16);
-        x[5] = __uint_as_float(q.z & 0xffff0000u);
-        x[6] = __uint_as_float(q.w << 16);
-        x[7] = __uint_as_float(q.w & 0xffff0000u);
-    }
+    static constexpr int kBytes = 2;
     static __device__ __forceinline__ float load1(const void *p)
     {
         return __uint_as_float((unsigned)__ldcs((const unsigned short *)p) << 16);
@@ -294,6 +281,12 @@ __device__ void scalar_step(DevState *st, const ScalarCfg &c, const Sched &sched
 
 // Persistent grid: every block walks its own segments and keeps two fp64 accumulators per
 // thread for the whole launch, so there is one block reduction and one partial pair per block.
+// Programmatic dependent launch: a kernel lets its successor in the stream be scheduled
+// early, and waits for its predecessor (completion and visibility of its writes) only where
+// it first depends on it.  Both are no-ops for a launch without the attribute.
+__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ unsigned smem_u32(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(u64 *bar, unsigned count)
@@ -424,8 +417,9 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     const int rps = S < kMaxRowsPerStage ? S : kMaxRowsPerStage;  // rows per stage
     const int n_chunks = (S + rps - 1) / rps;
     const unsigned stage_bytes = (unsigned)rps * kRowBytes;
-    const long long n_tiles = a.tprefix[T];
+    const long long n_tiles = a.n_tiles;
 
+    griddep_launch();
     if (tid == 0) {
         for (int i = 0; i < kStages; ++i) {
             mbar_init(&full_bar[i], 1);
@@ -440,7 +434,6 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     double accD = 0.0, accN = 0.0;
     unsigned item = 0;  // running count of staged work items, identical in every thread
     bool timed_out = false;
-    int k = 0;          // tensor that holds the current tile; tiles only move forward
 
     if (producer) {
         u64 policy;
@@ -448,17 +441,25 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
         int last_use[kStages];
 #pragma unroll
         for (int i = 0; i < kStages; ++i) last_use[i] = -1;
-        int held = -1;      // tensor whose row pointer this lane holds (row = lane, when S <= 32)
-        const char *rowptr = nullptr;
-        for (long long t = blockIdx.x; t < n_tiles && !timed_out; t += gridDim.x) {
-            while (t >= a.tprefix[k + 1]) ++k;
-            const long long c0 = (t - a.tprefix[k]) * kTile;
-            const long long cols = a.numel[k] & ~7LL;
-            const int tc = cols - c0 < kTile ? (int)(cols - c0) : kTile;
-            if (held != k) {
-                held = k;
-                if (lane < S) rowptr = (const char *)a.gptr[(size_t)lane * T + k];
-            }
+        // Round-robin tiles make every block visit most tensors, so table misses must stay off
+        // the copy queue: the descriptor is fetched two tiles ahead and this lane's row pointer
+        // (row = lane when S <= 32) one tile ahead.
+        const long long G = gridDim.x;
+        TileDesc d0, d1 = {}, d2 = {};
+        const char *rowptr = nullptr, *rowptr_n = nullptr;
+        if ((long long)blockIdx.x < n_tiles) d1 = a.tiles[blockIdx.x];
+        if ((long long)blockIdx.x + G < n_tiles) d2 = a.tiles[blockIdx.x + G];
+        if ((long long)blockIdx.x < n_tiles && lane < S) rowptr_n = (const char *)a.gptr[(size_t)lane * T + d1.tensor];
+        for (long long t = blockIdx.x; t < n_tiles && !timed_out; t += G) {
+            d0 = d1;
+            rowptr = rowptr_n;
+            d1 = d2;
+            if (t + 2 * G < n_tiles) d2 = a.tiles[t + 2 * G];
+            if (t + G < n_tiles && d1.tensor != d0.tensor && lane < S)
+                rowptr_n = (const char *)a.gptr[(size_t)lane * T + d1.tensor];
+            const int k = d0.tensor;
+            const long long c0 = d0.first;
+            const int tc = d0.len;
             for (int ch = 0; ch < n_chunks; ++ch, ++item) {
                 const int st = item % kStages;
                 const unsigned use = item / kStages;
@@ -492,12 +493,18 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                 if (last_use[i] >= 0) mbar_wait(&full_bar[i], (unsigned)last_use[i] & 1u);
         }
     } else {
+        // The producer above may already stream gradient rows while the previous kernel in the
+        // stream (the update that still reads the old mean gradient) drains; nothing may be
+        // written before it has finished.
+        griddep_wait();
         float c[CPT], s1[CPT], s2[CPT], p1[CPT], x[CPT];
-        for (long long t = blockIdx.x; t < n_tiles && !timed_out; t += gridDim.x) {
-            while (t >= a.tprefix[k + 1]) ++k;
-            const long long c0 = (t - a.tprefix[k]) * kTile;
-            const long long cols = a.numel[k] & ~7LL;
-            const int tc = cols - c0 < kTile ? (int)(cols - c0) : kTile;
+        const long long G = gridDim.x;
+        TileDesc d0, d1 = {};  // descriptor one tile ahead, as above
+        if ((long long)blockIdx.x < n_tiles) d1 = a.tiles[blockIdx.x];
+        for (long long t = blockIdx.x; t < n_tiles && !timed_out; t += G) {
+            d0 = d1;
+            if (t + G < n_tiles) d1 = a.tiles[t + G];
+            const int tc = d0.len;
             const bool active = tid * CPT < tc;
             for (int ch = 0; ch < n_chunks; ++ch, ++item) {
                 const int st = item % kStages;
@@ -554,26 +561,20 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                         dacc += fmaf(-q, s1[j], s2[j]);
                         nacc = fmaf(m[j], m[j], nacc);
                     }
-                    store_cols<CPT>(a.gbar + a.goff[k] + c0 + tid * CPT, m);
+                    store_cols<CPT>(a.gbar + d0.goff + tid * CPT, m);
                     accD += (double)dacc;
                     accN += (double)nacc;
                 }
             }
         }
         // ragged tails (< 8 elements) and tensors that are not 16-byte aligned: plain loads
-        const long long n_stiles = a.sprefix[T];
-        int k2 = 0;
-        for (long long t = blockIdx.x; t < n_stiles; t += gridDim.x) {
-            while (t >= a.sprefix[k2 + 1]) ++k2;
-            const long long n = a.numel[k2];
-            const long long start = (a.gflags[k2] & 1u) ? (n & ~7LL) : 0;
-            const long long first = start + (t - a.sprefix[k2]) * kScalarTile;
-            const int len = n - first < kScalarTile ? (int)(n - first) : kScalarTile;
-            float *gb = a.gbar + a.goff[k2] + first;
-            for (int e = tid; e < len; e += kThreads) {
-                float d, nn;
-                column_scalar<DT>(a.gptr, T, k2, ((size_t)first + e) * E, S, a.fS, gb + e, d, nn);
-                accD += (double)d;
+        for (long long t = blockIdx.x; t < a.n_stiles; t += gridDim.x) {
+            const TileDesc d = a.stiles[t];
+            float *gb = a.gbar + d.goff;
+            for (int e = tid; e < d.len; e += kThreads) {
+                float dd, nn;
+                column_scalar<DT>(a.gptr, T, d.tensor, ((size_t)d.first + e) * E, S, a.fS, gb + e, dd, nn);
+                accD += (double)dd;
                 accN += (double)nn;
             }
         }
@@ -625,29 +626,37 @@ __device__ __forceinline__ void update4(float4 &ww, float4 &vv, const float4 &gg
 
 __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const __grid_constant__ UpdateArgs a)
 {
+    griddep_launch();
+    griddep_wait();  // eta_t and the mean gradient come from the reduce kernel just before
     if (a.st->status & ADASCALE_STATUS_NONFINITE) return;
     const float eta = (float)a.st->eta;
     const int tid = threadIdx.x, T = a.T;
-    const long long n_tiles = a.uprefix[T];
-    int k = 0, held = -1;
-    float *wp = nullptr, *vp = nullptr;
-    const float *gp = nullptr;
-    long long n = 0;
-    bool vec = false;
-    for (long long t = blockIdx.x; t < n_tiles; t += gridDim.x) {
-        while (t >= a.uprefix[k + 1]) ++k;
-        if (k != held) {  // tiles only move forward, so a tensor's pointers are fetched once
-            held = k;
-            wp = (float *)a.wv[k];
-            vp = (float *)a.wv[T + k];
-            gp = a.gbar + a.goff[k];
-            n = a.numel[k];
-            vec = (a.wflags[k] & 1u) != 0;
+    const long long n_tiles = a.n_tiles, G = gridDim.x;
+    // descriptor two tiles ahead, the tensor's pointers one tile ahead (see the reduce kernel)
+    TileDesc d0, d1 = {}, d2 = {};
+    float *wp = nullptr, *vp = nullptr, *wp_n = nullptr, *vp_n = nullptr;
+    unsigned fl = 0, fl_n = 0;
+    if ((long long)blockIdx.x < n_tiles) {
+        d1 = a.tiles[blockIdx.x];
+        wp_n = (float *)a.wv[d1.tensor];
+        vp_n = (float *)a.wv[T + d1.tensor];
+        fl_n = a.wflags[d1.tensor];
+    }
+    if ((long long)blockIdx.x + G < n_tiles) d2 = a.tiles[blockIdx.x + G];
+    for (long long t = blockIdx.x; t < n_tiles; t += G) {
+        d0 = d1; wp = wp_n; vp = vp_n; fl = fl_n;
+        d1 = d2;
+        if (t + 2 * G < n_tiles) d2 = a.tiles[t + 2 * G];
+        if (t + G < n_tiles && d1.tensor != d0.tensor) {
+            wp_n = (float *)a.wv[d1.tensor];
+            vp_n = (float *)a.wv[T + d1.tensor];
+            fl_n = a.wflags[d1.tensor];
         }
-        const long long first = (t - a.uprefix[k]) * kUpdateTile;
-        const int len = n - first < kUpdateTile ? (int)(n - first) : kUpdateTile;
+        const long long first = d0.first;
+        const int len = d0.len;
         float *w = wp + first, *v = vp + first;
-        const float *g = gp + first;
+        const float *g = a.gbar + d0.goff;
+        const bool vec = (fl & 1u) != 0;
         if (vec && len == kUpdateTile) {
             const float4 gg = ((const float4 *)g)[tid];
             float4 ww = ((const float4 *)w)[tid];
@@ -745,17 +754,18 @@ struct adascale_ctx {
     unsigned flags = 0;
     std::vector<long long> numel;
     std::vector<long long> goff;
-    std::vector<long long> uprefix;
     long long P = 0, gbar_elems = 0;
-    long long *d_numel = nullptr, *d_goff = nullptr, *d_uprefix = nullptr;
+    TileDesc *d_rtiles = nullptr;   // reduce kernel: staged tiles, then scalar tiles
+    TileDesc *d_utiles = nullptr;   // update kernel
+    long long rtiles_cap = 0, n_utiles = 0;
+    std::vector<unsigned char> tiled_aligned;  // alignment flags and tile width the device descriptors were built for
+    int tiled_cpt = 0;
     float *d_gbar = nullptr;
     double2 *d_partials = nullptr;
     unsigned *d_ticket = nullptr;
     DevState *d_state = nullptr;
     PtrTable tg, tw;
-    // tiling of the last reduce table
-    int cpt = 0;
-    long long n_tiles = 0, n_stiles = 0;
+    long long n_tiles = 0, n_stiles = 0;  // of the descriptors on the device
     DevState *h_snap = nullptr;  // pinned
     cudaEvent_t ev_snap = nullptr;
     bool snap_inflight = false;
@@ -852,6 +862,33 @@ void build_prefixes(const long long *numel, const unsigned char *aligned, int T,
     sprefix[T] = ns;
 }
 
+// Descriptors of the reduce kernel's tiles: all staged tiles in tensor order, then all
+// scalar-path tiles.
+void build_reduce_tiles(const long long *numel, const long long *goff, const unsigned char *aligned, int T,
+                        int tile_cols, std::vector<TileDesc> &out, long long &n_staged)
+{
+    out.clear();
+    auto emit = [&](int k, long long first, long long len) {
+        TileDesc d = {};
+        d.first = first;
+        d.goff = goff[k] + first;
+        d.tensor = k;
+        d.len = (int)len;
+        out.push_back(d);
+    };
+    for (int k = 0; k < T; ++k) {
+        if (aligned && !aligned[k]) continue;
+        const long long cols = numel[k] & ~7LL;
+        for (long long c0 = 0; c0 < cols; c0 += tile_cols) emit(k, c0, cols - c0 < tile_cols ? cols - c0 : tile_cols);
+    }
+    n_staged = (long long)out.size();
+    for (int k = 0; k < T; ++k) {
+        const long long n = numel[k];
+        const long long start = (!aligned || aligned[k]) ? (n & ~7LL) : 0;
+        for (long long f = start; f < n; f += kScalarTile) emit(k, f, n - f < kScalarTile ? n - f : kScalarTile);
+    }
+}
+
 // ---- pointer tables ----------------------------------------------------------------------
 
 adascale_status table_alloc(adascale_ctx *ctx, PtrTable &t, size_t words)
@@ -900,6 +937,24 @@ adascale_status table_sync(adascale_ctx *ctx, PtrTable &t, const std::vector<u64
 
 // ---- launches ----------------------------------------------------------------------------
 
+// Launch that may overlap its prologue with the tail of the previous kernel in the stream.
+template <typename Args>
+cudaError_t launch_overlapped(void (*kernel)(Args), int n_blocks, int threads, size_t smem, cudaStream_t s,
+                              const Args &a)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)n_blocks);
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, a);
+}
+
 template <int DT, int CPT>
 cudaError_t launch_reduce_one(int n_blocks, const ReduceArgs &a, size_t smem, cudaStream_t s)
 {
@@ -912,8 +967,7 @@ cudaError_t launch_reduce_one(int n_blocks, const ReduceArgs &a, size_t smem, cu
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    k_reduce<DT, CPT><<<dim3(n_blocks), dim3(kStagedThreads), smem, s>>>(a);
-    return cudaGetLastError();
+    return launch_overlapped(k_reduce<DT, CPT>, n_blocks, kStagedThreads, smem, s, a);
 }
 
 cudaError_t launch_reduce(int dtype, int cpt, int n_blocks, const ReduceArgs &a, size_t smem, cudaStream_t s)
@@ -939,17 +993,14 @@ bool valid_sched(const adascale_lr_schedule *s)
     return true;
 }
 
-// Layout of the reduce table in 8-byte words:
-//   [max_S * T row pointers][T + 1 staged-tile prefix][T + 1 scalar-tile prefix][ceil(T/2) flags]
+// Layout of the reduce table in 8-byte words: [max_S * T row pointers]
 adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const adascale_lr_schedule *sched,
                           cudaStream_t s)
 {
     const int S = ctx->S, T = ctx->T;
     const size_t esz = ctx->dtype == ADASCALE_BF16 ? 2 : 4;
-    const size_t w_ptr = 0, w_tp = (size_t)ctx->max_S * T, w_sp = w_tp + T + 1, w_fl = w_sp + T + 1;
     std::vector<u64> fresh(ctx->tg.words, 0);
     std::vector<unsigned char> aligned((size_t)T, 1);
-    unsigned *flags = reinterpret_cast<unsigned *>(fresh.data() + w_fl);
     for (int k = 0; k < T; ++k) {
         for (int i = 0; i < S; ++i) {
             const u64 p = (u64)(uintptr_t)grads[(size_t)i * T + k];
@@ -958,27 +1009,44 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
                 if (p % esz) return ADASCALE_ERR_ALIGNMENT;
                 if (p % 16) aligned[k] = 0;
             }
-            fresh[w_ptr + (size_t)i * T + k] = p;
+            fresh[(size_t)i * T + k] = p;
         }
-        flags[k] = aligned[k];
     }
     const int max_blocks = ctx->sms * kReduceBlocksPerSM;
     const int cpt = choose_cpt(ctx->dtype, S, ctx->numel.data(), aligned.data(), T, max_blocks);
-    build_prefixes(ctx->numel.data(), aligned.data(), T, kThreads * cpt,
-                   reinterpret_cast<long long *>(fresh.data() + w_tp),
-                   reinterpret_cast<long long *>(fresh.data() + w_sp));
-    const long long n_tiles = (long long)fresh[w_tp + T], n_stiles = (long long)fresh[w_sp + T];
+    if (cpt != ctx->tiled_cpt || aligned != ctx->tiled_aligned) {
+        // the tiling follows the tile width (a function of S) and the alignment of the pointers
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        CU(cudaStreamIsCapturing(s, &cap));
+        if (cap != cudaStreamCaptureStatusNone) {
+            ctx->err = "tiling changed inside a stream capture";
+            return ADASCALE_ERR_STATE;
+        }
+        std::vector<TileDesc> tiles;
+        long long n_staged = 0;
+        build_reduce_tiles(ctx->numel.data(), ctx->goff.data(), aligned.data(), T, kThreads * cpt, tiles, n_staged);
+        if ((long long)tiles.size() > ctx->rtiles_cap) return ADASCALE_ERR_TOO_LARGE;  // cannot happen: sized for the worst case
+        if (!tiles.empty()) {
+            // pageable source: the runtime stages it before the call returns
+            CU(cudaMemcpyAsync(ctx->d_rtiles, tiles.data(), tiles.size() * sizeof(TileDesc), cudaMemcpyHostToDevice, s));
+            CU(cudaStreamSynchronize(s));
+        }
+        ctx->n_tiles = n_staged;
+        ctx->n_stiles = (long long)tiles.size() - n_staged;
+        ctx->tiled_cpt = cpt;
+        ctx->tiled_aligned = aligned;
+    }
     adascale_status st = table_sync(ctx, ctx->tg, fresh, s);
     if (st != ADASCALE_OK) return st;
+    const long long n_tiles = ctx->n_tiles, n_stiles = ctx->n_stiles;
     if (n_tiles + n_stiles == 0) return ADASCALE_OK;  // nothing but empty tensors
 
     ReduceArgs a;
-    a.gptr = ctx->tg.dev + w_ptr;
-    a.tprefix = reinterpret_cast<const long long *>(ctx->tg.dev + w_tp);
-    a.sprefix = reinterpret_cast<const long long *>(ctx->tg.dev + w_sp);
-    a.gflags = reinterpret_cast<const unsigned *>(ctx->tg.dev + w_fl);
-    a.numel = ctx->d_numel;
-    a.goff = ctx->d_goff;
+    a.gptr = ctx->tg.dev;
+    a.tiles = ctx->d_rtiles;
+    a.stiles = ctx->d_rtiles + n_tiles;
+    a.n_tiles = n_tiles;
+    a.n_stiles = n_stiles;
     a.gbar = ctx->d_gbar;
     a.partials = ctx->d_partials;
     a.ticket = ctx->d_ticket;
@@ -1003,9 +1071,6 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
     const size_t smem = (size_t)kStages * rows_per_stage(S) * kThreads * cpt * esz;
     cudaError_t e = launch_reduce(ctx->dtype, cpt, (int)nb, a, smem, s);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "launch of the reduce kernel");
-    ctx->cpt = cpt;
-    ctx->n_tiles = n_tiles;
-    ctx->n_stiles = n_stiles;
     ctx->launches += 1;
     ctx->reduced = true;
     ctx->last_stream = s;
@@ -1030,15 +1095,14 @@ adascale_status do_update(adascale_ctx *ctx, void *const *params, void *const *m
     }
     adascale_status st = table_sync(ctx, ctx->tw, fresh, s);
     if (st != ADASCALE_OK) return st;
-    const long long n_tiles = ctx->uprefix[(size_t)T];
+    const long long n_tiles = ctx->n_utiles;
     if (n_tiles == 0) return ADASCALE_OK;
 
     UpdateArgs a;
     a.wv = ctx->tw.dev;
     a.wflags = reinterpret_cast<const unsigned *>(ctx->tw.dev + (size_t)2 * T);
-    a.uprefix = ctx->d_uprefix;
-    a.numel = ctx->d_numel;
-    a.goff = ctx->d_goff;
+    a.tiles = ctx->d_utiles;
+    a.n_tiles = n_tiles;
     a.gbar = ctx->d_gbar;
     a.st = ctx->d_state;
     a.T = T;
@@ -1046,8 +1110,7 @@ adascale_status do_update(adascale_ctx *ctx, void *const *params, void *const *m
     a.lambda = (float)ctx->lambda;
     long long nb = n_tiles;
     if (nb > (long long)ctx->sms * kUpdateBlocksPerSM) nb = (long long)ctx->sms * kUpdateBlocksPerSM;
-    k_update<<<dim3((unsigned)nb), dim3(kThreads), 0, s>>>(a);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_overlapped(k_update, (int)nb, kThreads, 0, s, a);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "launch of the update kernel");
     ctx->launches += 1;
     ctx->last_stream = s;
@@ -1146,29 +1209,38 @@ adascale_status adascale_init(const adascale_config *cfg, adascale_ctx **out)
     ctx->flags = cfg->flags;
     ctx->numel.assign(cfg->numel, cfg->numel + cfg->n_tensors);
 
-    long long g = 0, ut = 0;
+    long long g = 0;
+    std::vector<TileDesc> utiles;
+    long long rcap = 0;  // worst case of the reduce tiling: everything unaligned, or the narrowest staged tile
     for (int k = 0; k < ctx->T; ++k) {
         const long long n = ctx->numel[k];
         ctx->goff.push_back(g);
-        ctx->uprefix.push_back(ut);
         ctx->P += n;
+        for (long long f = 0; f < n; f += kUpdateTile) {
+            TileDesc d = {};
+            d.first = f;
+            d.goff = g + f;
+            d.tensor = k;
+            d.len = (int)(n - f < kUpdateTile ? n - f : kUpdateTile);
+            utiles.push_back(d);
+        }
+        const long long narrow = kThreads * 8 / 4;  // 8 bytes per thread and row of fp32
+        rcap += (n + narrow - 1) / narrow + 1;
         g += (n + kGbarAlign - 1) / kGbarAlign * kGbarAlign;
-        ut += (n + kUpdateTile - 1) / kUpdateTile;
     }
-    ctx->uprefix.push_back(ut);
     ctx->gbar_elems = g;
+    ctx->n_utiles = (long long)utiles.size();
+    ctx->rtiles_cap = rcap;
 
     DeviceGuard guard(ctx->device);
     auto body = [&]() -> adascale_status {
         if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
         CU(cudaDeviceGetAttribute(&ctx->sms, cudaDevAttrMultiProcessorCount, ctx->device));
         const size_t T = (size_t)ctx->T;
-        CU(cudaMalloc(&ctx->d_numel, T * sizeof(long long)));
-        CU(cudaMalloc(&ctx->d_goff, T * sizeof(long long)));
-        CU(cudaMalloc(&ctx->d_uprefix, (T + 1) * sizeof(long long)));
-        CU(cudaMemcpy(ctx->d_numel, ctx->numel.data(), T * sizeof(long long), cudaMemcpyHostToDevice));
-        CU(cudaMemcpy(ctx->d_goff, ctx->goff.data(), T * sizeof(long long), cudaMemcpyHostToDevice));
-        CU(cudaMemcpy(ctx->d_uprefix, ctx->uprefix.data(), (T + 1) * sizeof(long long), cudaMemcpyHostToDevice));
+        CU(cudaMalloc(&ctx->d_rtiles, (size_t)(rcap > 0 ? rcap : 1) * sizeof(TileDesc)));
+        CU(cudaMalloc(&ctx->d_utiles, (utiles.empty() ? 1 : utiles.size()) * sizeof(TileDesc)));
+        if (!utiles.empty())
+            CU(cudaMemcpy(ctx->d_utiles, utiles.data(), utiles.size() * sizeof(TileDesc), cudaMemcpyHostToDevice));
         CU(cudaMalloc(&ctx->d_gbar, (size_t)(g > 0 ? g : 1) * sizeof(float)));
         CU(cudaMemset(ctx->d_gbar, 0, (size_t)(g > 0 ? g : 1) * sizeof(float)));
         CU(cudaMalloc(&ctx->d_partials, (size_t)(ctx->sms * kReduceBlocksPerSM + 1) * sizeof(double2)));
@@ -1176,7 +1248,7 @@ adascale_status adascale_init(const adascale_config *cfg, adascale_ctx **out)
         CU(cudaMemset(ctx->d_ticket, 0, sizeof(unsigned)));
         CU(cudaMalloc(&ctx->d_state, sizeof(DevState)));
         CU(cudaMemset(ctx->d_state, 0, sizeof(DevState)));
-        adascale_status s1 = table_alloc(ctx, ctx->tg, (size_t)ctx->max_S * T + 2 * (T + 1) + (T + 1) / 2);
+        adascale_status s1 = table_alloc(ctx, ctx->tg, (size_t)ctx->max_S * T);
         if (s1 != ADASCALE_OK) return s1;
         s1 = table_alloc(ctx, ctx->tw, 2 * T + (T + 1) / 2);
         if (s1 != ADASCALE_OK) return s1;
@@ -1200,9 +1272,8 @@ adascale_status adascale_destroy(adascale_ctx *ctx)
     DeviceGuard guard(ctx->device);
     if (guard.ok) {
         cudaDeviceSynchronize();
-        cudaFree(ctx->d_numel);
-        cudaFree(ctx->d_goff);
-        cudaFree(ctx->d_uprefix);
+        cudaFree(ctx->d_rtiles);
+        cudaFree(ctx->d_utiles);
         cudaFree(ctx->d_gbar);
         cudaFree(ctx->d_partials);
         cudaFree(ctx->d_ticket);
