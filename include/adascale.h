@@ -226,6 +226,41 @@ adascale_status adascale_tiling(const int64_t *numel, int32_t n_tensors, int32_t
                                 const uint8_t *aligned, int32_t n_blocks, int64_t *tprefix, int64_t *sprefix,
                                 int32_t *tile_cols, int32_t *rows);
 
+/*
+ * The two sums and the mean gradient of ONE tensor without any allocation (the paper has no
+ * counterpart; the sums are those of App. B.3 in the form the reduce kernel uses:
+ * sums[0] = sum_i ||g_i - gbar||^2, sums[1] = ||gbar||^2).
+ *
+ * Who needs it: every other entry point works on a context, and adascale_init calls
+ * cudaMalloc.  That is no use to a caller that is not allowed to allocate device memory: a
+ * component that runs after start-up in a process where all device memory has already been
+ * handed to another allocator, or one that must never risk the late failure or the implicit
+ * device synchronisation that an allocation can bring.  Such a caller brings its own buffers
+ * for inputs and outputs; what the kernel needs beyond them (a table of the row pointers,
+ * a counter, one pair of partial sums per block, about 17 KB) sits in a fixed array inside
+ * the library that every GPU which loads the library holds until the process exits.  The
+ * call makes no cudaMalloc, cudaFree or other allocating call.
+ *
+ *   rows        host array [S] of device pointers, 16-byte aligned, n elements of grad_dtype each
+ *   S           1 .. ADASCALE_STATIC_MAX_ROWS
+ *   n           1 .. ADASCALE_STATIC_MAX_NUMEL
+ *   gbar        device pointer, n float32, 16-byte aligned: receives the mean gradient
+ *   sums        device pointer, 2 float64, 8-byte aligned: receives the two sums
+ *   cuda_stream stream of the current device; the call enqueues and returns
+ * Larger S or n: ADASCALE_ERR_TOO_LARGE ("size beyond the documented maximum"); null or bad
+ * dtype: INVALID_ARG; misaligned pointers: ALIGNMENT; a failing CUDA call: ERR_CUDA.
+ *
+ * The first call on a device looks up the array's device address and the device's size; make
+ * that first call outside of any stream capture.  All calls on a device share the one array
+ * and it keeps what the last call left there (the call resets what has to start at zero), so
+ * two calls that can overlap on the GPU - different streams without an ordering between them,
+ * or different host threads - race on it and give wrong results; order them.
+ */
+#define ADASCALE_STATIC_MAX_ROWS 32
+#define ADASCALE_STATIC_MAX_NUMEL 2147483640LL
+adascale_status adascale_grad_stats_static(const void *const *rows, int32_t S, int32_t grad_dtype, int64_t n,
+                                           void *gbar, void *sums, void *cuda_stream);
+
 /* Number of kernels the library has launched through this context since init. */
 int64_t adascale_launch_count(const adascale_ctx *ctx);
 

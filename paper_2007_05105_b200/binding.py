@@ -22,7 +22,7 @@ STATE_BYTES = 128
 
 EXPORTS = ("adascale_init", "adascale_step", "adascale_reduce", "adascale_update", "adascale_get_gain_tau",
            "adascale_mean_grad", "adascale_set_scale", "adascale_get_state", "adascale_set_state",
-           "adascale_step_host", "adascale_stream_probe", "adascale_tiling", "adascale_launch_count",
+           "adascale_step_host", "adascale_stream_probe", "adascale_tiling", "adascale_grad_stats_static", "adascale_launch_count",
            "adascale_destroy",
            "adascale_strerror", "adascale_last_error")
 
@@ -75,6 +75,7 @@ def _load():
     L.adascale_tiling.argtypes = [C.POINTER(C.c_int64), C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_uint8),
                                   C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int32),
                                   C.POINTER(C.c_int32)]
+    L.adascale_grad_stats_static.argtypes = [vpp, C.c_int32, C.c_int32, C.c_int64, vp, vp, vp]
     L.adascale_launch_count.argtypes = [vp]
     L.adascale_launch_count.restype = C.c_int64
     L.adascale_destroy.argtypes = [vp]
@@ -252,6 +253,24 @@ def tiling(numels, S, grad_dtype="f32", aligned=None, n_blocks=296):
     if status != OK:
         raise AdaScaleError(status, strerror(status))
     return list(tp), list(sp), cols.value, rows.value
+
+
+STATIC_MAX_ROWS = 32
+STATIC_MAX_NUMEL = 2147483640
+
+
+def grad_stats_static(rows, n, grad_dtype, gbar, sums, stream=None, device=0):
+    """Mean gradient and the two sums of one tensor through the entry point that allocates nothing.
+
+    For callers that may not allocate device memory: rows, gbar (float32, n) and sums
+    (float64, 2) are the caller's buffers; the library's own scratch is a fixed array.  Calls
+    that can overlap on the GPU share that array and must be ordered by the caller.
+    """
+    s = C.c_void_p(_current_stream(device) if stream is None else int(stream))
+    status = lib.adascale_grad_stats_static(pointer_array(rows), len(rows), {"f32": F32, "bf16": BF16}.get(grad_dtype, grad_dtype),
+                                            int(n), C.c_void_p(_ptr(gbar)), C.c_void_p(_ptr(sums)), s)
+    if status != OK:
+        raise AdaScaleError(status, strerror(status))
 
 
 def stream_probe(kind, a, b, n_bytes, stream=None, device=0):

@@ -22,6 +22,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -684,6 +685,121 @@ __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const _
                 w[e] = fmaf(-eta, vn, w[e]);
             }
         }
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Allocation-free variant of the reduce kernel for one tensor: the same shifted sums, the
+// same fp64 partials and fixed-order second stage, but rows are read with plain 128-bit loads
+// and everything the kernel needs besides its inputs and outputs (row-pointer table, ticket,
+// per-block partials) lives in one file-scope device array instead of memory from cudaMalloc.
+// ---------------------------------------------------------------------------------------
+constexpr int kStaticMaxRows = ADASCALE_STATIC_MAX_ROWS;
+constexpr int kStaticMaxBlocks = 1024;
+constexpr size_t kStaticPtrBytes = 256;     // 32 row pointers
+constexpr size_t kStaticTicketOff = 256;    // one counter, padded to 256 bytes
+constexpr size_t kStaticPartialOff = 512;   // kStaticMaxBlocks pairs of doubles
+constexpr size_t kStaticScratchBytes = kStaticPartialOff + kStaticMaxBlocks * sizeof(double2);
+
+// Shared by every call on this device and kept until the process exits (about 17 KB).
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+struct StaticArgs {
+    unsigned char *scratch;  // device address of g_static_scratch, resolved on the host
+    float *gbar;
+    double *sums;            // [0] = sum_i ||g_i - gbar||^2, [1] = ||gbar||^2
+    long long n;
+    int S;
+    float invS, fS;
+};
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads) k_grad_stats_static(const __grid_constant__ StaticArgs a)
+{
+    __shared__ double sa[kWarps], sb[kWarps];
+    __shared__ bool is_last;
+    constexpr int E = Elem<DT>::kBytes;
+    constexpr int V = 8;  // columns per thread and step
+    const u64 *rows = reinterpret_cast<const u64 *>(a.scratch);
+    unsigned *ticket = reinterpret_cast<unsigned *>(a.scratch + kStaticTicketOff);
+    double2 *partials = reinterpret_cast<double2 *>(a.scratch + kStaticPartialOff);
+    const int tid = threadIdx.x, S = a.S;
+    const long long nv = a.n / V;
+    double accD = 0.0, accN = 0.0;
+
+    for (long long v = (long long)blockIdx.x * kThreads + tid; v < nv; v += (long long)gridDim.x * kThreads) {
+        const size_t boff = (size_t)v * V * E;
+        float c[V], s1[V], s2[V], p1[V], x[V];
+        if (S >= 3) {  // shift = median of the first three rows
+            float x1[V], x2[V];
+            Cols<DT, V>::load((const char *)rows[0] + boff, x);
+            Cols<DT, V>::load((const char *)rows[1] + boff, x1);
+            Cols<DT, V>::load((const char *)rows[2] + boff, x2);
+#pragma unroll
+            for (int j = 0; j < V; ++j) {
+                const float lo = fminf(x[j], x1[j]), hi = fmaxf(x[j], x1[j]);
+                c[j] = fmaxf(lo, fminf(hi, x2[j]));
+            }
+        } else {
+            Cols<DT, V>::load((const char *)rows[0] + boff, c);
+        }
+#pragma unroll
+        for (int j = 0; j < V; ++j) s1[j] = s2[j] = 0.f;
+        for (int r = 0; r < S; r += 8) {  // s1 in blocks of 8 rows
+#pragma unroll
+            for (int j = 0; j < V; ++j) p1[j] = 0.f;
+            for (int rr = r; rr < S && rr < r + 8; ++rr) {
+                Cols<DT, V>::load((const char *)rows[rr] + boff, x);
+                accumulate_row<V>(x, c, p1, s2);
+            }
+#pragma unroll
+            for (int j = 0; j < V; ++j) s1[j] += p1[j];
+        }
+        float m[V];
+        float dacc = 0.f, nacc = 0.f;
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+            float q = s1[j] * a.invS;
+            const float res = fmaf(-q, a.fS, s1[j]);
+            q = fmaf(res, a.invS, q);
+            m[j] = c[j] + q;
+            dacc += fmaf(-q, s1[j], s2[j]);
+            nacc = fmaf(m[j], m[j], nacc);
+        }
+        store_cols<V>(a.gbar + v * V, m);
+        accD += (double)dacc;
+        accN += (double)nacc;
+    }
+    if (blockIdx.x == 0) {  // ragged tail, fewer than 8 elements
+        for (long long e = nv * V + tid; e < a.n; e += kThreads) {
+            float d, nn;
+            column_scalar<DT>(rows, 1, 0, (size_t)e * E, S, a.fS, a.gbar + e, d, nn);
+            accD += (double)d;
+            accN += (double)nn;
+        }
+    }
+
+    block_sum2<kWarps>(accD, accN, sa, sb);
+    if (tid == 0) {
+        partials[blockIdx.x] = make_double2(accD, accN);
+        __threadfence();
+        const unsigned tk = atomicAdd(ticket, 1u);
+        is_last = (tk == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    double d = 0.0, n = 0.0;
+    for (int i = tid; i < (int)gridDim.x; i += kThreads) {
+        const double2 p = __ldcg(&partials[i]);
+        d += p.x;
+        n += p.y;
+    }
+    block_sum2<kWarps>(d, n, sa, sb);
+    if (tid == 0) {
+        a.sums[0] = d;
+        a.sums[1] = n;
+        *ticket = 0u;
     }
 }
 
@@ -1509,6 +1625,69 @@ adascale_status adascale_stream_probe(int32_t kind, void *a, void *b, int64_t n_
     } else {
         k_probe_rmw<<<(unsigned)blocks, kThreads, 0, s>>>((float4 *)a, (const float4 *)b, n);
     }
+    CU(cudaGetLastError());
+    return ADASCALE_OK;
+}
+
+adascale_status adascale_grad_stats_static(const void *const *rows, int32_t S, int32_t grad_dtype, int64_t n,
+                                           void *gbar, void *sums, void *cuda_stream)
+{
+    adascale_ctx *ctx = nullptr;  // for the CU macro: there is no context here
+    if (!rows || !gbar || !sums || S < 1 || n < 1) return ADASCALE_ERR_INVALID_ARG;
+    if (grad_dtype != ADASCALE_F32 && grad_dtype != ADASCALE_BF16) return ADASCALE_ERR_INVALID_ARG;
+    if (S > kStaticMaxRows || n > ADASCALE_STATIC_MAX_NUMEL) return ADASCALE_ERR_TOO_LARGE;
+    for (int i = 0; i < S; ++i) {
+        if (!rows[i]) return ADASCALE_ERR_INVALID_ARG;
+        if ((uintptr_t)rows[i] % 16) return ADASCALE_ERR_ALIGNMENT;
+    }
+    if (((uintptr_t)gbar % 16) || ((uintptr_t)sums % 8)) return ADASCALE_ERR_ALIGNMENT;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+
+    // Set-up, once per device and with that device current: in host code the array's name is
+    // only a handle, the address a kernel can use comes from cudaGetSymbolAddress.
+    static std::mutex mu;
+    static unsigned char *scratch_of[64] = {nullptr};
+    static int sms_of[64] = {0};
+    int dev = 0;
+    CU(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return ADASCALE_ERR_INVALID_ARG;
+    unsigned char *scratch = nullptr;
+    int sms = 0;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!scratch_of[dev]) {
+            void *p = nullptr;
+            CU(cudaGetSymbolAddress(&p, g_static_scratch));
+            CU(cudaDeviceGetAttribute(&sms_of[dev], cudaDevAttrMultiProcessorCount, dev));
+            scratch_of[dev] = static_cast<unsigned char *>(p);
+        }
+        scratch = scratch_of[dev];
+        sms = sms_of[dev];
+    }
+
+    // the row pointers go into the scratch array; the ticket must start at zero whatever the
+    // previous call left behind
+    u64 table[kStaticMaxRows] = {0};
+    for (int i = 0; i < S; ++i) table[i] = (u64)(uintptr_t)rows[i];
+    CU(cudaMemcpyAsync(scratch, table, kStaticPtrBytes, cudaMemcpyHostToDevice, s));  // pageable: staged before return
+    CU(cudaMemsetAsync(scratch + kStaticTicketOff, 0, sizeof(unsigned), s));
+
+    StaticArgs a;
+    a.scratch = scratch;
+    a.gbar = static_cast<float *>(gbar);
+    a.sums = static_cast<double *>(sums);
+    a.n = n;
+    a.S = S;
+    a.fS = (float)S;
+    a.invS = 1.0f / (float)S;
+    long long blocks = (n / 8 + kThreads - 1) / kThreads;
+    const long long cap = (long long)sms * 8 < kStaticMaxBlocks ? (long long)sms * 8 : kStaticMaxBlocks;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    if (grad_dtype == ADASCALE_BF16)
+        k_grad_stats_static<ADASCALE_BF16><<<(unsigned)blocks, kThreads, 0, s>>>(a);
+    else
+        k_grad_stats_static<ADASCALE_F32><<<(unsigned)blocks, kThreads, 0, s>>>(a);
     CU(cudaGetLastError());
     return ADASCALE_OK;
 }
