@@ -129,6 +129,12 @@ def max_over_ranks(value, world, device=None):
     return float(t.item())
 
 
+def whole_job_value(local_ms, step_bytes, world, device=None):
+    """(slowest rank's ms per step, GB/s summed over the replicas at that pace)."""
+    ms = max_over_ranks(local_ms, world, device)
+    return ms, world * step_bytes / (ms * 1e-3) / 1e9
+
+
 def barrier(world):
     if world > 1:
         import torch.distributed as dist
@@ -275,8 +281,7 @@ def run_ours(args, wl):
     barrier(world)
     torch.cuda.synchronize(dev)
     clocks = sampler.stop() if rank == 0 else None
-    ms_per_step = max_over_ranks(local_ms, world, dev)
-    value = world * step_b / (ms_per_step * 1e-3) / 1e9
+    ms_per_step, value = whole_job_value(local_ms, step_b, world, dev)
 
     # ---- per-kernel timing (separate pass: events between the two launches of a step)
     ksteps = min(steps, 200)
