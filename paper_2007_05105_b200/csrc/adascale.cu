@@ -325,6 +325,104 @@ __device__ __forceinline__ void bulk_load(void *dst, const void *src, unsigned b
                  : "memory");
 }
 
+// ---- packed fp32 pairs -------------------------------------------------------------------
+// sm_100 adds, subtracts and multiply-adds two fp32 values with one instruction (f32x2).  The
+// consumer loop of the reduce kernel keeps its per-column state in such pairs: same IEEE
+// operations in the same order as scalar code, half the instruction issue.
+typedef unsigned long long f2;
+
+__device__ __forceinline__ f2 pack2(float lo, float hi)
+{
+    f2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f2 v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f2 add2(f2 a, f2 b)
+{
+    f2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f2 sub2(f2 a, f2 b)
+{
+    f2 r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f2 fma2(f2 a, f2 b, f2 c)
+{
+    f2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+// a bf16 pair in one 32-bit word -> two fp32 (widening is a shift / a mask, exact)
+__device__ __forceinline__ f2 widen2(unsigned u)
+{
+    f2 r;
+    asm("{\n\t.reg .b32 lo, hi;\n\tshl.b32 lo, %1, 16;\n\tand.b32 hi, %1, 0xffff0000;\n\tmov.b64 %0, {lo, hi};\n\t}"
+        : "=l"(r)
+        : "r"(u));
+    return r;
+}
+
+// CPT columns of one staged row, from shared memory (32-bit shared address plus a
+// compile-time byte offset), as CPT/2 packed pairs.
+template <int DT, int CPT> struct PairLoad;
+template <int CPT> struct PairLoad<ADASCALE_F32, CPT> {
+    template <int OFF>
+    static __device__ __forceinline__ void load(unsigned addr, f2 *x)
+    {
+        if constexpr (CPT == 2) {
+            asm volatile("ld.shared.b64 %0, [%1+%2];" : "=l"(x[0]) : "r"(addr), "n"(OFF));
+        } else {
+#pragma unroll
+            for (int k = 0; k < CPT / 4; ++k)
+                asm volatile("ld.shared.v2.b64 {%0, %1}, [%2+%3];"
+                             : "=l"(x[2 * k]), "=l"(x[2 * k + 1])
+                             : "r"(addr + 16 * k), "n"(OFF));
+        }
+    }
+};
+template <int CPT> struct PairLoad<ADASCALE_BF16, CPT> {
+    template <int OFF>
+    static __device__ __forceinline__ void load(unsigned addr, f2 *x)
+    {
+        if constexpr (CPT == 4) {
+            unsigned u0, u1;
+            asm volatile("ld.shared.v2.b32 {%0, %1}, [%2+%3];" : "=r"(u0), "=r"(u1) : "r"(addr), "n"(OFF));
+            x[0] = widen2(u0);
+            x[1] = widen2(u1);
+        } else {
+            unsigned u0, u1, u2, u3;
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4+%5];"
+                         : "=r"(u0), "=r"(u1), "=r"(u2), "=r"(u3)
+                         : "r"(addr), "n"(OFF));
+            x[0] = widen2(u0);
+            x[1] = widen2(u1);
+            x[2] = widen2(u2);
+            x[3] = widen2(u3);
+        }
+    }
+};
+
+// One staged row into the running sums: d = x - c, p1 += d, s2 += d * d.
+template <int DT, int CPT, int OFF>
+__device__ __forceinline__ void consume_row(unsigned addr, const f2 *c, f2 *p1, f2 *s2)
+{
+    f2 x[CPT / 2];
+    PairLoad<DT, CPT>::template load<OFF>(addr, x);
+#pragma unroll
+    for (int j = 0; j < CPT / 2; ++j) {
+        const f2 d = sub2(x[j], c[j]);
+        p1[j] = add2(p1[j], d);
+        s2[j] = fma2(d, d, s2[j]);
+    }
+}
+
 template <int DT, int CPT> struct Cols;
 template <int CPT> struct Cols<ADASCALE_F32, CPT> {
     static __device__ __forceinline__ void load(const char *p, float *x)
@@ -498,10 +596,12 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
         // stream (the update that still reads the old mean gradient) drains; nothing may be
         // written before it has finished.
         griddep_wait();
-        float c[CPT], s1[CPT], s2[CPT], p1[CPT], x[CPT];
+        constexpr int NP = CPT / 2;
+        f2 c[NP], s1[NP], s2[NP], p1[NP];  // per-column state as packed pairs
         const long long G = gridDim.x;
         TileDesc d0, d1 = {};  // descriptor one tile ahead, as above
         if ((long long)blockIdx.x < n_tiles) d1 = a.tiles[blockIdx.x];
+        const unsigned lane_base = smem_u32(stage_mem) + (unsigned)tid * CPT * E;
         for (long long t = blockIdx.x; t < n_tiles && !timed_out; t += G) {
             d0 = d1;
             if (t + G < n_tiles) d1 = a.tiles[t + G];
@@ -513,37 +613,55 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                 if (!mbar_wait(&full_bar[st], use & 1u)) { timed_out = true; break; }
                 const int r0 = ch * rps;
                 const int rows = S - r0 < rps ? S - r0 : rps;
-                const char *base = (const char *)stage_mem + (size_t)st * stage_bytes + (size_t)tid * CPT * E;
+                unsigned addr = lane_base + (unsigned)st * stage_bytes;
                 if (active) {
                     if (ch == 0) {
                         if (S >= 3) {  // shift = median of the first three rows
-                            float x1[CPT], x2[CPT];
-                            Cols<DT, CPT>::load(base, x);
-                            Cols<DT, CPT>::load(base + kRowBytes, x1);
-                            Cols<DT, CPT>::load(base + 2 * kRowBytes, x2);
+                            f2 x0[NP], x1[NP], x2[NP];
+                            PairLoad<DT, CPT>::template load<0>(addr, x0);
+                            PairLoad<DT, CPT>::template load<kRowBytes>(addr, x1);
+                            PairLoad<DT, CPT>::template load<2 * kRowBytes>(addr, x2);
 #pragma unroll
-                            for (int j = 0; j < CPT; ++j) {
-                                const float lo = fminf(x[j], x1[j]), hi = fmaxf(x[j], x1[j]);
-                                c[j] = fmaxf(lo, fminf(hi, x2[j]));
+                            for (int j = 0; j < NP; ++j) {
+                                float a0, a1, b0, b1, e0, e1;
+                                unpack2(x0[j], a0, a1);
+                                unpack2(x1[j], b0, b1);
+                                unpack2(x2[j], e0, e1);
+                                const float m0 = fmaxf(fminf(a0, b0), fminf(fmaxf(a0, b0), e0));
+                                const float m1 = fmaxf(fminf(a1, b1), fminf(fmaxf(a1, b1), e1));
+                                c[j] = pack2(m0, m1);
                             }
                         } else {
-                            Cols<DT, CPT>::load(base, c);
+                            PairLoad<DT, CPT>::template load<0>(addr, c);
                         }
 #pragma unroll
-                        for (int j = 0; j < CPT; ++j) s1[j] = s2[j] = 0.f;
+                        for (int j = 0; j < NP; ++j) s1[j] = s2[j] = 0ull;  // +0.0f, +0.0f
                     }
-                    for (int r = 0; r < rows; r += 8) {
+                    int r = 0;
+                    for (; r + 8 <= rows; r += 8) {  // s1 in blocks of 8 rows
 #pragma unroll
-                        for (int j = 0; j < CPT; ++j) p1[j] = 0.f;
+                        for (int j = 0; j < NP; ++j) p1[j] = 0ull;
+                        consume_row<DT, CPT, 0 * kRowBytes>(addr, c, p1, s2);
+                        consume_row<DT, CPT, 1 * kRowBytes>(addr, c, p1, s2);
+                        consume_row<DT, CPT, 2 * kRowBytes>(addr, c, p1, s2);
+                        consume_row<DT, CPT, 3 * kRowBytes>(addr, c, p1, s2);
+                        consume_row<DT, CPT, 4 * kRowBytes>(addr, c, p1, s2);
+                        consume_row<DT, CPT, 5 * kRowBytes>(addr, c, p1, s2);
+                        consume_row<DT, CPT, 6 * kRowBytes>(addr, c, p1, s2);
+                        consume_row<DT, CPT, 7 * kRowBytes>(addr, c, p1, s2);
 #pragma unroll
-                        for (int rr = 0; rr < 8; ++rr) {
-                            if (r + rr < rows) {
-                                Cols<DT, CPT>::load(base + (size_t)(r + rr) * kRowBytes, x);
-                                accumulate_row<CPT>(x, c, p1, s2);
-                            }
+                        for (int j = 0; j < NP; ++j) s1[j] = add2(s1[j], p1[j]);
+                        addr += 8 * kRowBytes;
+                    }
+                    if (r < rows) {
+#pragma unroll
+                        for (int j = 0; j < NP; ++j) p1[j] = 0ull;
+                        for (; r < rows; ++r) {
+                            consume_row<DT, CPT, 0>(addr, c, p1, s2);
+                            addr += kRowBytes;
                         }
 #pragma unroll
-                        for (int j = 0; j < CPT; ++j) s1[j] += p1[j];
+                        for (int j = 0; j < NP; ++j) s1[j] = add2(s1[j], p1[j]);
                     }
                 }
                 __syncwarp();
@@ -552,15 +670,22 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                     float m[CPT];
                     float dacc = 0.f, nacc = 0.f;
 #pragma unroll
-                    for (int j = 0; j < CPT; ++j) {
-                        // quotient s1/S: reciprocal multiply plus one residual correction (1/S is not
-                        // exact unless S is a power of two, and a biased 1/S would bias every column alike)
-                        float q = s1[j] * a.invS;
-                        const float res = fmaf(-q, a.fS, s1[j]);
-                        q = fmaf(res, a.invS, q);
-                        m[j] = c[j] + q;
-                        dacc += fmaf(-q, s1[j], s2[j]);
-                        nacc = fmaf(m[j], m[j], nacc);
+                    for (int j = 0; j < NP; ++j) {
+                        float cc[2], ss1[2], ss2[2];
+                        unpack2(c[j], cc[0], cc[1]);
+                        unpack2(s1[j], ss1[0], ss1[1]);
+                        unpack2(s2[j], ss2[0], ss2[1]);
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            // quotient s1/S: reciprocal multiply plus one residual correction (1/S is not
+                            // exact unless S is a power of two, and a biased 1/S would bias every column alike)
+                            float q = ss1[h] * a.invS;
+                            const float res = fmaf(-q, a.fS, ss1[h]);
+                            q = fmaf(res, a.invS, q);
+                            m[2 * j + h] = cc[h] + q;
+                            dacc += fmaf(-q, ss1[h], ss2[h]);
+                            nacc = fmaf(m[2 * j + h], m[2 * j + h], nacc);
+                        }
                     }
                     store_cols<CPT>(a.gbar + d0.goff + tid * CPT, m);
                     accD += (double)dacc;
