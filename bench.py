@@ -24,6 +24,9 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "adascale_step gradient GB/s and % of B200 HBM peak; step latency (us)"
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the reduce kernel, from the ncu
+# captures summarised under profiles/ (same kernel build); None where no capture exists
+NCU_TRAFFIC_BYTES = {"resnet18": 382.5e6, "resnet50": 875.4e6}
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 L2_BYTES = 126 * 1024 * 1024
@@ -374,7 +377,7 @@ def run_ours(args, wl):
                        else ("inputs larger than L2 (working set %d MB)" % (working_set >> 20)),
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "roofline": {"bound": "hbm", "kernel": "k_reduce", "achieved": reduce_gbs, "peak": peak, "unit": "GB/s",
-                         "frac": reduce_gbs / peak, "peak_kind": peak_kind + " copy bandwidth", "traffic": None,
+                         "frac": reduce_gbs / peak, "peak_kind": peak_kind + " copy bandwidth", "traffic": NCU_TRAFFIC_BYTES.get(wl.name),
                          "bytes_per_launch": reduce_b, "us_per_launch": t_reduce * 1e3,
                          "update_kernel": {"kernel": "k_update", "achieved": update_gbs, "frac": update_gbs / peak,
                                            "bytes_per_launch": update_b, "us_per_launch": t_update * 1e3}},
