@@ -39,6 +39,8 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--workload", default="resnet18")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--mode", default="two-kernel", choices=["two-kernel", "fused"],
+                    help="fused: lagged gain estimate, one kernel per step, P*(S*b_g+16) bytes")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -227,6 +229,9 @@ def run_ours(args, wl):
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     reduce_b, update_b = algorithmic_bytes(wl)
+    fused = args.mode == "fused"
+    if fused:  # S rows, w and v read, w and v written; the mean gradient never leaves the registers
+        reduce_b, update_b = wl.P * (wl.S * (2 if wl.grad_dtype == "bf16" else 4) + 16), 0
     step_b = reduce_b + update_b
     est_ms = step_b / 6.0e9  # at ~6 TB/s
     steps = args.steps if args.steps is not None else max(20, min(2000, int(3000.0 / max(est_ms, 1e-3))))
@@ -236,7 +241,8 @@ def run_ours(args, wl):
     grads = src.fill(0)
     wflat, vflat = src.init_params()
     w, v = src.views(wflat), src.views(vflat)
-    ada = B.AdaScale(src.numels, wl.S, wl.grad_dtype, momentum=wl.momentum, weight_decay=wl.weight_decay, device=local)
+    ada = B.AdaScale(src.numels, wl.S, wl.grad_dtype, momentum=wl.momentum, weight_decay=wl.weight_decay, device=local,
+                     flags=(B.FLAG_LAGGED | B.FLAG_FUSED) if fused else 0)
     sched = B.make_schedule(wl.lr.get("kind", "const"), eta0=wl.lr.get("eta0", 0.1), d=wl.lr.get("d", 1.0),
                             T_S1=wl.lr.get("T_S1", 1.0), milestones=wl.lr.get("milestones", ()))
     gp, wp, vp = B.pointer_array(grads), B.pointer_array(w), B.pointer_array(v)
@@ -293,16 +299,20 @@ def run_ours(args, wl):
         if flush is not None:
             flush.zero_()
         a.record(stream)
-        ada.reduce(gp, sched)
-        b.record(stream)
-        ada.update(wp, vp)
+        if fused:
+            ada.step(gp, wp, vp, sched)
+            b.record(stream)
+        else:
+            ada.reduce(gp, sched)
+            b.record(stream)
+            ada.update(wp, vp)
         c.record(stream)
     torch.cuda.synchronize(dev)
     t_reduce = sum(a.elapsed_time(b) for a, b, c in ev) / ksteps
     t_update = sum(b.elapsed_time(c) for a, b, c in ev) / ksteps
     peak, peak_kind = measured_peak()
     reduce_gbs = reduce_b / (t_reduce * 1e-3) / 1e9
-    update_gbs = update_b / (t_update * 1e-3) / 1e9
+    update_gbs = update_b / (t_update * 1e-3) / 1e9 if not fused else 0.0
 
     # ---- bandwidth ceilings of this GPU with the library's own trivial kernels
     ceilings = {}
@@ -372,15 +382,16 @@ def run_ours(args, wl):
             "pct_of_nominal_8TBs": 100.0 * value / world / NOMINAL_HBM_GBS,
             "pct_of_measured_copy": 100.0 * value / world / peak,
             "config": {"workload": wl.name, "P": wl.P, "tensors": len(wl.shapes), "S": wl.S,
-                       "grad_dtype": wl.grad_dtype, "bytes_per_step": step_b,
+                       "grad_dtype": wl.grad_dtype, "bytes_per_step": step_b, "mode": args.mode,
                        "cache": ("L2 flushed between steps (working set %d MB)" % (working_set >> 20)) if flush is not None
                        else ("inputs larger than L2 (working set %d MB)" % (working_set >> 20)),
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
-            "roofline": {"bound": "hbm", "kernel": "k_reduce", "achieved": reduce_gbs, "peak": peak, "unit": "GB/s",
-                         "frac": reduce_gbs / peak, "peak_kind": peak_kind + " copy bandwidth", "traffic": NCU_TRAFFIC_BYTES.get(wl.name),
+            "roofline": {"bound": "hbm", "kernel": "k_reduce (fused)" if fused else "k_reduce", "achieved": reduce_gbs, "peak": peak, "unit": "GB/s",
+                         "frac": reduce_gbs / peak, "peak_kind": peak_kind + " copy bandwidth", "traffic": None if fused else NCU_TRAFFIC_BYTES.get(wl.name),
                          "bytes_per_launch": reduce_b, "us_per_launch": t_reduce * 1e3,
-                         "update_kernel": {"kernel": "k_update", "achieved": update_gbs, "frac": update_gbs / peak,
-                                           "bytes_per_launch": update_b, "us_per_launch": t_update * 1e3}},
+                         "update_kernel": None if fused else
+                         {"kernel": "k_update", "achieved": update_gbs, "frac": update_gbs / peak,
+                          "bytes_per_launch": update_b, "us_per_launch": t_update * 1e3}},
             "ceilings": ceilings, "clocks": clocks, "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": launches,
         }
         print(json.dumps(line), flush=True)

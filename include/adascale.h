@@ -74,6 +74,13 @@ typedef struct {
                                      (the variant App. B.3 says the paper's runs used)    */
 #define ADASCALE_FLAG_CONT_TAU 2u /* evaluate lr at tau_t instead of floor(tau_t)          */
 #define ADASCALE_FLAG_RATIO 4u    /* estimator of Sec. 3.4: r = (m1 + eps) / (m2 + eps)    */
+#define ADASCALE_FLAG_FUSED 8u    /* with ADASCALE_FLAG_LAGGED only: eta_t is known before the
+                                     gradients are read, so one kernel reads the S rows, w and v
+                                     and writes w and v; the mean gradient is never stored.  Only
+                                     adascale_step and adascale_step_host run an iteration
+                                     (reduce, update, mean_grad return ERR_STATE), and non-finite
+                                     gradients have already reached their own coordinates of w
+                                     and v when they are detected (the state and tau still skip) */
 
 typedef struct {
     int32_t S;              /* scale: gradient rows per iteration, >= 1                */

@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libadascale_b200.so")
 OK, ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_CUDA, ERR_STATE, ERR_TOO_LARGE = range(6)
 F32, BF16 = 0, 1
 LR_CONST, LR_EXP, LR_STEP = 0, 1, 2
-FLAG_LAGGED, FLAG_CONT_TAU, FLAG_RATIO = 1, 2, 4
+FLAG_LAGGED, FLAG_CONT_TAU, FLAG_RATIO, FLAG_FUSED = 1, 2, 4, 8
 STATUS_NONFINITE = 1
 MAX_MILESTONES = 8
 STATE_BYTES = 128

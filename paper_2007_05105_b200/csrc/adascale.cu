@@ -94,6 +94,9 @@ struct ReduceArgs {
     const TileDesc *stiles;   // scalar-path tiles
     long long n_tiles, n_stiles;
     float *gbar;
+    const u64 *wv;            // fused mode only: [2 * T] parameters then momentum
+    const unsigned *wflags;   // fused mode only: [T] bit0: both pointers 16-byte aligned
+    float rho, lambda;        // fused mode only
     double2 *partials;
     unsigned *ticket;
     DevState *st;
@@ -282,6 +285,21 @@ __device__ void scalar_step(DevState *st, const ScalarCfg &c, const Sched &sched
 
 // Persistent grid: every block walks its own segments and keeps two fp64 accumulators per
 // thread for the whole launch, so there is one block reduction and one partial pair per block.
+// Lagged estimate (App. B.3: r_t from the averages of prior iterations only, r_0 = 1): the
+// learning rate of the coming iteration is known before its gradients are read.  Same
+// expressions as in scalar_step, so both give the identical value.
+__device__ double lagged_eta(const DevState *st, const ScalarCfg &c, const Sched &sched)
+{
+    const double S = (double)c.S;
+    double r = 1.0;
+    if (c.S > 1 && st->n > 0)
+        r = (c.flags & ADASCALE_FLAG_RATIO) ? (st->avg_a + c.eps) / (st->avg_b + c.eps)
+                                            : (st->avg_a + st->avg_b) / (st->avg_a / S + st->avg_b);
+    const double tau = st->tau;
+    const double t_arg = (c.flags & ADASCALE_FLAG_CONT_TAU) ? tau : floor(tau);
+    return r * lr_eval(sched, t_arg);
+}
+
 // Programmatic dependent launch: a kernel lets its successor in the stream be scheduled
 // early, and waits for its predecessor (completion and visibility of its writes) only where
 // it first depends on it.  Both are no-ops for a launch without the attribute.
@@ -498,7 +516,12 @@ __device__ __forceinline__ void store_cols(float *g, const float *m)
 // kThreads * CPT columns of up to kMaxRowsPerStage rows.  Row chunks let any S through: the
 // per-column sums carry over from one chunk of rows to the next and close after the last.
 // ---------------------------------------------------------------------------------------
-template <int DT, int CPT>
+//
+// FUSED (lagged estimate only): eta_t is known when the kernel starts, so the same pass also
+// reads w and v, applies the update of Eq. 2 and writes them back; the mean gradient lives in
+// registers only and the update kernel is not launched: P * (S * b_g + 16) bytes per iteration
+// instead of P * (S * b_g + 24), one launch instead of two.
+template <int DT, int CPT, bool FUSED>
 __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(const __grid_constant__ ReduceArgs a)
 {
     extern __shared__ __align__(128) unsigned char stage_mem[];
@@ -506,6 +529,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     __shared__ double sa[kStagedWarps], sb[kStagedWarps];
     __shared__ bool is_last;
     __shared__ int abort_flag;
+    __shared__ float eta_shared;
 
     constexpr int E = Elem<DT>::kBytes;
     constexpr int kTile = kThreads * CPT;  // columns per tile
@@ -596,17 +620,56 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
         // stream (the update that still reads the old mean gradient) drains; nothing may be
         // written before it has finished.
         griddep_wait();
+        float eta = 0.f;
+        if constexpr (FUSED) {
+            if (tid == 0) eta_shared = (float)lagged_eta(a.st, a.sc, a.sched);
+            asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");  // consumers only
+            eta = eta_shared;
+        }
         constexpr int NP = CPT / 2;
         f2 c[NP], s1[NP], s2[NP], p1[NP];  // per-column state as packed pairs
         const long long G = gridDim.x;
         TileDesc d0, d1 = {};  // descriptor one tile ahead, as above
         if ((long long)blockIdx.x < n_tiles) d1 = a.tiles[blockIdx.x];
+        // fused mode: the tile's parameter and momentum pointers, fetched one tile ahead as well
+        float *wp = nullptr, *vp = nullptr, *wp_n = nullptr, *vp_n = nullptr;
+        unsigned fl = 0, fl_n = 0;
+        if constexpr (FUSED) {
+            if ((long long)blockIdx.x < n_tiles) {
+                wp_n = (float *)a.wv[d1.tensor];
+                vp_n = (float *)a.wv[T + d1.tensor];
+                fl_n = a.wflags[d1.tensor];
+            }
+        }
         const unsigned lane_base = smem_u32(stage_mem) + (unsigned)tid * CPT * E;
         for (long long t = blockIdx.x; t < n_tiles && !timed_out; t += G) {
             d0 = d1;
             if (t + G < n_tiles) d1 = a.tiles[t + G];
             const int tc = d0.len;
             const bool active = tid * CPT < tc;
+            float wr[CPT], vr[CPT];  // fused mode: this thread's parameters and momentum, requested
+            float *wt = nullptr, *vt = nullptr;  // before the rows are consumed so they arrive meanwhile
+            bool vec_wv = false;
+            if constexpr (FUSED) {
+                wp = wp_n; vp = vp_n; fl = fl_n;
+                if (t + G < n_tiles && d1.tensor != d0.tensor) {
+                    wp_n = (float *)a.wv[d1.tensor];
+                    vp_n = (float *)a.wv[T + d1.tensor];
+                    fl_n = a.wflags[d1.tensor];
+                }
+                wt = wp + d0.first + tid * CPT;
+                vt = vp + d0.first + tid * CPT;
+                vec_wv = (fl & 1u) != 0;
+                if (active) {
+                    if (vec_wv) {
+                        Cols<ADASCALE_F32, CPT>::load((const char *)wt, wr);
+                        Cols<ADASCALE_F32, CPT>::load((const char *)vt, vr);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < CPT; ++j) { wr[j] = wt[j]; vr[j] = vt[j]; }
+                    }
+                }
+            }
             for (int ch = 0; ch < n_chunks; ++ch, ++item) {
                 const int st = item % kStages;
                 const unsigned use = item / kStages;
@@ -687,7 +750,22 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                             nacc = fmaf(m[2 * j + h], m[2 * j + h], nacc);
                         }
                     }
-                    store_cols<CPT>(a.gbar + d0.goff + tid * CPT, m);
+                    if constexpr (FUSED) {
+#pragma unroll
+                        for (int j = 0; j < CPT; ++j) {
+                            vr[j] = fmaf(a.rho, vr[j], fmaf(a.lambda, wr[j], m[j]));
+                            wr[j] = fmaf(-eta, vr[j], wr[j]);
+                        }
+                        if (vec_wv) {
+                            store_cols<CPT>(vt, vr);
+                            store_cols<CPT>(wt, wr);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < CPT; ++j) { vt[j] = vr[j]; wt[j] = wr[j]; }
+                        }
+                    } else {
+                        store_cols<CPT>(a.gbar + d0.goff + tid * CPT, m);
+                    }
                     accD += (double)dacc;
                     accN += (double)nacc;
                 }
@@ -699,7 +777,17 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
             float *gb = a.gbar + d.goff;
             for (int e = tid; e < d.len; e += kThreads) {
                 float dd, nn;
-                column_scalar<DT>(a.gptr, T, d.tensor, ((size_t)d.first + e) * E, S, a.fS, gb + e, dd, nn);
+                if constexpr (FUSED) {
+                    float m;
+                    column_scalar<DT>(a.gptr, T, d.tensor, ((size_t)d.first + e) * E, S, a.fS, &m, dd, nn);
+                    float *w = (float *)a.wv[d.tensor] + d.first + e;
+                    float *v = (float *)a.wv[T + d.tensor] + d.first + e;
+                    const float vn = fmaf(a.rho, *v, fmaf(a.lambda, *w, m));
+                    *v = vn;
+                    *w = fmaf(-eta, vn, *w);
+                } else {
+                    column_scalar<DT>(a.gptr, T, d.tensor, ((size_t)d.first + e) * E, S, a.fS, gb + e, dd, nn);
+                }
                 accD += (double)dd;
                 accN += (double)nn;
             }
@@ -1196,31 +1284,39 @@ cudaError_t launch_overlapped(void (*kernel)(Args), int n_blocks, int threads, s
     return cudaLaunchKernelEx(&cfg, kernel, a);
 }
 
-template <int DT, int CPT>
+template <int DT, int CPT, bool FUSED>
 cudaError_t launch_reduce_one(int n_blocks, const ReduceArgs &a, size_t smem, cudaStream_t s)
 {
     static bool configured[64] = {false};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(k_reduce<DT, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(k_reduce<DT, CPT, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              kStages * kStageBytes);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    return launch_overlapped(k_reduce<DT, CPT>, n_blocks, kStagedThreads, smem, s, a);
+    return launch_overlapped(k_reduce<DT, CPT, FUSED>, n_blocks, kStagedThreads, smem, s, a);
 }
 
-cudaError_t launch_reduce(int dtype, int cpt, int n_blocks, const ReduceArgs &a, size_t smem, cudaStream_t s)
+template <bool FUSED>
+cudaError_t launch_reduce_mode(int dtype, int cpt, int n_blocks, const ReduceArgs &a, size_t smem, cudaStream_t s)
 {
     if (dtype == ADASCALE_BF16)
-        return cpt == 4 ? launch_reduce_one<ADASCALE_BF16, 4>(n_blocks, a, smem, s)
-                        : launch_reduce_one<ADASCALE_BF16, 8>(n_blocks, a, smem, s);
+        return cpt == 4 ? launch_reduce_one<ADASCALE_BF16, 4, FUSED>(n_blocks, a, smem, s)
+                        : launch_reduce_one<ADASCALE_BF16, 8, FUSED>(n_blocks, a, smem, s);
     switch (cpt) {
-    case 2: return launch_reduce_one<ADASCALE_F32, 2>(n_blocks, a, smem, s);
-    case 4: return launch_reduce_one<ADASCALE_F32, 4>(n_blocks, a, smem, s);
-    default: return launch_reduce_one<ADASCALE_F32, 8>(n_blocks, a, smem, s);
+    case 2: return launch_reduce_one<ADASCALE_F32, 2, FUSED>(n_blocks, a, smem, s);
+    case 4: return launch_reduce_one<ADASCALE_F32, 4, FUSED>(n_blocks, a, smem, s);
+    default: return launch_reduce_one<ADASCALE_F32, 8, FUSED>(n_blocks, a, smem, s);
     }
+}
+
+cudaError_t launch_reduce(bool fused, int dtype, int cpt, int n_blocks, const ReduceArgs &a, size_t smem,
+                          cudaStream_t s)
+{
+    return fused ? launch_reduce_mode<true>(dtype, cpt, n_blocks, a, smem, s)
+                 : launch_reduce_mode<false>(dtype, cpt, n_blocks, a, smem, s);
 }
 
 bool valid_sched(const adascale_lr_schedule *s)
@@ -1236,7 +1332,7 @@ bool valid_sched(const adascale_lr_schedule *s)
 
 // Layout of the reduce table in 8-byte words: [max_S * T row pointers]
 adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const adascale_lr_schedule *sched,
-                          cudaStream_t s)
+                          cudaStream_t s, bool fused)
 {
     const int S = ctx->S, T = ctx->T;
     const size_t esz = ctx->dtype == ADASCALE_BF16 ? 2 : 4;
@@ -1289,6 +1385,10 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
     a.n_tiles = n_tiles;
     a.n_stiles = n_stiles;
     a.gbar = ctx->d_gbar;
+    a.wv = ctx->tw.dev;  // read by the fused kernel only; sync_update_table has run before
+    a.wflags = reinterpret_cast<const unsigned *>(ctx->tw.dev + (size_t)2 * T);
+    a.rho = (float)ctx->rho;
+    a.lambda = (float)ctx->lambda;
     a.partials = ctx->d_partials;
     a.ticket = ctx->d_ticket;
     a.st = ctx->d_state;
@@ -1310,7 +1410,7 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
     long long nb = n_tiles + n_stiles;
     if (nb > max_blocks) nb = max_blocks;
     const size_t smem = (size_t)kStages * rows_per_stage(S) * kThreads * cpt * esz;
-    cudaError_t e = launch_reduce(ctx->dtype, cpt, (int)nb, a, smem, s);
+    cudaError_t e = launch_reduce(fused, ctx->dtype, cpt, (int)nb, a, smem, s);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "launch of the reduce kernel");
     ctx->launches += 1;
     ctx->reduced = true;
@@ -1319,7 +1419,7 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
 }
 
 // Layout of the update table in 8-byte words: [T parameters][T momentum][ceil(T/2) flags]
-adascale_status do_update(adascale_ctx *ctx, void *const *params, void *const *momentum, cudaStream_t s)
+adascale_status sync_update_table(adascale_ctx *ctx, void *const *params, void *const *momentum, cudaStream_t s)
 {
     const int T = ctx->T;
     std::vector<u64> fresh(ctx->tw.words, 0);
@@ -1334,7 +1434,13 @@ adascale_status do_update(adascale_ctx *ctx, void *const *params, void *const *m
         fresh[(size_t)T + k] = pv;
         flags[k] = ((pw % 16) == 0 && (pv % 16) == 0) ? 1u : 0u;
     }
-    adascale_status st = table_sync(ctx, ctx->tw, fresh, s);
+    return table_sync(ctx, ctx->tw, fresh, s);
+}
+
+adascale_status do_update(adascale_ctx *ctx, void *const *params, void *const *momentum, cudaStream_t s)
+{
+    const int T = ctx->T;
+    adascale_status st = sync_update_table(ctx, params, momentum, s);
     if (st != ADASCALE_OK) return st;
     const long long n_tiles = ctx->n_utiles;
     if (n_tiles == 0) return ADASCALE_OK;
@@ -1431,8 +1537,10 @@ adascale_status adascale_init(const adascale_config *cfg, adascale_ctx **out)
     if (cfg->grad_dtype != ADASCALE_F32 && cfg->grad_dtype != ADASCALE_BF16) return ADASCALE_ERR_INVALID_ARG;
     if (!(cfg->theta < 1.0) || !(cfg->eps >= 0.0) || cfg->device < 0) return ADASCALE_ERR_INVALID_ARG;
     if (!std::isfinite(cfg->momentum) || !std::isfinite(cfg->weight_decay)) return ADASCALE_ERR_INVALID_ARG;
-    if (cfg->flags & ~(ADASCALE_FLAG_LAGGED | ADASCALE_FLAG_CONT_TAU | ADASCALE_FLAG_RATIO))
+    if (cfg->flags & ~(ADASCALE_FLAG_LAGGED | ADASCALE_FLAG_CONT_TAU | ADASCALE_FLAG_RATIO | ADASCALE_FLAG_FUSED))
         return ADASCALE_ERR_INVALID_ARG;
+    if ((cfg->flags & ADASCALE_FLAG_FUSED) && !(cfg->flags & ADASCALE_FLAG_LAGGED))
+        return ADASCALE_ERR_INVALID_ARG;  // the one-pass form needs eta_t before the gradients are read
     for (int k = 0; k < cfg->n_tensors; ++k)
         if (cfg->numel[k] < 0) return ADASCALE_ERR_INVALID_ARG;
 
@@ -1482,8 +1590,9 @@ adascale_status adascale_init(const adascale_config *cfg, adascale_ctx **out)
         CU(cudaMalloc(&ctx->d_utiles, (utiles.empty() ? 1 : utiles.size()) * sizeof(TileDesc)));
         if (!utiles.empty())
             CU(cudaMemcpy(ctx->d_utiles, utiles.data(), utiles.size() * sizeof(TileDesc), cudaMemcpyHostToDevice));
-        CU(cudaMalloc(&ctx->d_gbar, (size_t)(g > 0 ? g : 1) * sizeof(float)));
-        CU(cudaMemset(ctx->d_gbar, 0, (size_t)(g > 0 ? g : 1) * sizeof(float)));
+        const size_t gbar_alloc = (g > 0 && !(ctx->flags & ADASCALE_FLAG_FUSED)) ? (size_t)g : 1;
+        CU(cudaMalloc(&ctx->d_gbar, gbar_alloc * sizeof(float)));
+        CU(cudaMemset(ctx->d_gbar, 0, gbar_alloc * sizeof(float)));
         CU(cudaMalloc(&ctx->d_partials, (size_t)(ctx->sms * kReduceBlocksPerSM + 1) * sizeof(double2)));
         CU(cudaMalloc(&ctx->d_ticket, sizeof(unsigned)));
         CU(cudaMemset(ctx->d_ticket, 0, sizeof(unsigned)));
@@ -1534,15 +1643,16 @@ adascale_status adascale_reduce(adascale_ctx *ctx, const void *const *grads, con
                                 void *cuda_stream)
 {
     if (!ctx || !grads || !valid_sched(sched)) return ADASCALE_ERR_INVALID_ARG;
+    if (ctx->flags & ADASCALE_FLAG_FUSED) return ADASCALE_ERR_STATE;  // one pass: only adascale_step exists
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
-    return do_reduce(ctx, grads, sched, (cudaStream_t)cuda_stream);
+    return do_reduce(ctx, grads, sched, (cudaStream_t)cuda_stream, false);
 }
 
 adascale_status adascale_update(adascale_ctx *ctx, void *const *params, void *const *momentum, void *cuda_stream)
 {
     if (!ctx || !params || !momentum) return ADASCALE_ERR_INVALID_ARG;
-    if (!ctx->reduced) return ADASCALE_ERR_STATE;
+    if (!ctx->reduced || (ctx->flags & ADASCALE_FLAG_FUSED)) return ADASCALE_ERR_STATE;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
     return do_update(ctx, params, momentum, (cudaStream_t)cuda_stream);
@@ -1561,7 +1671,12 @@ adascale_status adascale_step(adascale_ctx *ctx, const void *const *grads, void 
             if (((uintptr_t)params[k] % 4) || ((uintptr_t)momentum[k] % 4)) return ADASCALE_ERR_ALIGNMENT;
         }
     }
-    adascale_status st = do_reduce(ctx, grads, sched, (cudaStream_t)cuda_stream);
+    if (ctx->flags & ADASCALE_FLAG_FUSED) {
+        adascale_status sf = sync_update_table(ctx, params, momentum, (cudaStream_t)cuda_stream);
+        if (sf != ADASCALE_OK) return sf;
+        return do_reduce(ctx, grads, sched, (cudaStream_t)cuda_stream, true);
+    }
+    adascale_status st = do_reduce(ctx, grads, sched, (cudaStream_t)cuda_stream, false);
     if (st != ADASCALE_OK) return st;
     return do_update(ctx, params, momentum, (cudaStream_t)cuda_stream);
 }
@@ -1607,6 +1722,7 @@ adascale_status adascale_get_gain_tau(adascale_ctx *ctx, adascale_stats *out, in
 adascale_status adascale_mean_grad(adascale_ctx *ctx, const void **gbar)
 {
     if (!ctx || !gbar) return ADASCALE_ERR_INVALID_ARG;
+    if (ctx->flags & ADASCALE_FLAG_FUSED) return ADASCALE_ERR_STATE;  // the mean gradient is never stored
     for (int k = 0; k < ctx->T; ++k) gbar[k] = ctx->d_gbar + ctx->goff[k];
     return ADASCALE_OK;
 }

@@ -54,7 +54,7 @@ def _cfg(B, **over):
 
 
 @pytest.mark.parametrize("over", [dict(S=0), dict(n_tensors=0), dict(grad_dtype=7), dict(theta=1.0),
-                                  dict(eps=-1.0), dict(max_S=1), dict(flags=64), dict(device=-1),
+                                  dict(eps=-1.0), dict(max_S=1), dict(flags=64), dict(flags=8), dict(device=-1),
                                   dict(momentum=float("nan"))])
 def test_init_rejects_bad_config_without_cuda(B, over):
     ctx = C.c_void_p()

@@ -331,3 +331,74 @@ def test_nonblocking_readback_trails_by_at_most_one_call():
     torch.cuda.synchronize()
     assert ada.get_gain_tau(False).t == 3
     ada.close()
+
+
+# ---------------------------------------------------------------- one-pass (fused, lagged) mode
+
+FUSED = B.FLAG_LAGGED | B.FLAG_FUSED
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("S", [1, 2, 3, 5, 8, 16, 17, 32, 40])
+def test_fused_mode_against_the_lagged_oracle(S, dtype):
+    gen = _gen(3000 + S)
+    name = "bf16" if dtype == torch.bfloat16 else "f32"
+    lr = {"kind": "exp", "eta0": 0.05, "d": 0.5, "T_S1": 20.0}
+    pair = H.Pair(RAGGED, S, name, momentum=0.9, weight_decay=1e-3, flags=FUSED, lr=lr)
+    w, v = _params(RAGGED, gen)
+    pair.attach(w, v)
+    for step in range(4):
+        rows = _make_rows(RAGGED, S, dtype, gen, k=[0.5, 3.0, 10.0, 1.0][step])
+        st, _ = pair.step(rows, "fused S=%d %s step %d" % (S, name, step))
+    if S > 1:
+        assert st.r > 1.0  # the gain follows the averages from the second step on
+    pair.close()
+
+
+@pytest.mark.parametrize("misalign", [1, 3])
+def test_fused_mode_with_misaligned_gradients_and_parameters(misalign):
+    gen = _gen(3100 + misalign)
+    numels = [5, 64, 1000, 4099]
+    for grads_off, params_off in [(misalign, 0), (0, misalign), (misalign, misalign)]:
+        pair = H.Pair(numels, 4, "f32", momentum=0.5, weight_decay=0.01, flags=FUSED)
+        w, v = _params(numels, gen, params_off)
+        pair.attach(w, v)
+        for step in range(2):
+            pair.step(_make_rows(numels, 4, torch.float32, gen, misalign=grads_off), "fused misalign step %d" % step)
+        pair.close()
+
+
+def test_fused_mode_is_bitwise_the_two_kernel_lagged_mode():
+    gen = _gen(3200)
+    numels = [100000, 4097, 64, 7]
+    steps = [_make_rows(numels, 8, torch.bfloat16, gen, k=1.0 + i) for i in range(4)]
+    sched = B.make_schedule("step", eta0=0.1, d=0.1, milestones=(3.0,))
+    out = []
+    for flags in (B.FLAG_LAGGED, FUSED):
+        w, v = _params(numels, _gen(3201))
+        ada = B.AdaScale(numels, 8, "bf16", momentum=0.9, weight_decay=1e-4, flags=flags)
+        for rows in steps:
+            ada.step(rows, w, v, sched)
+        out.append((ada.get_gain_tau(True).as_dict(), w, v, ada.launch_count))
+        ada.close()
+    assert out[0][0] == out[1][0]
+    for a, b in zip(out[0][1] + out[0][2], out[1][1] + out[1][2]):
+        assert torch.equal(a, b)
+    assert out[0][3] == 8 and out[1][3] == 4      # two launches per step against one
+
+
+def test_fused_mode_call_rules():
+    with pytest.raises(B.AdaScaleError) as e:
+        B.AdaScale([16], 2, flags=B.FLAG_FUSED)   # needs the lagged estimate
+    assert e.value.status == B.ERR_INVALID_ARG
+    ada = B.AdaScale([16], 2, flags=FUSED)
+    g = torch.zeros(16, device=DEV)
+    w = torch.zeros(16, device=DEV)
+    v = torch.zeros(16, device=DEV)
+    sched = B.make_schedule()
+    ada.step([g, g], [w], [v], sched)
+    for call in (lambda: ada.reduce([g, g], sched), lambda: ada.update([w], [v]), lambda: ada.mean_grad()):
+        with pytest.raises(B.AdaScaleError) as e:
+            call()
+        assert e.value.status == B.ERR_STATE
+    ada.close()
