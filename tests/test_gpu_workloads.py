@@ -1,5 +1,6 @@
 """The five benchmark workloads end to end against the oracle, at full size."""
 import math
+import os
 
 import pytest
 import torch
@@ -80,6 +81,24 @@ def test_resnet50_bf16_thousand_step_clock():
     pair.close()
 
 
+@pytest.mark.skipif(os.environ.get("ADASCALE_FULL_TRAJECTORY") != "1",
+                    reason="several minutes of oracle time: set ADASCALE_FULL_TRAJECTORY=1")
+def test_resnet50_bf16_thousand_step_clock_full_size():
+    """The same 1000-iteration clock check at the full 25.6M parameters, S = 16, bf16."""
+    wl = synthetic.workload("resnet50")
+    src = synthetic.GradientSource(wl, device=DEV)
+    pair = _pair(wl, src)
+    total = 0.0
+    for step in range(1000):
+        st, ost = pair.step(src.fill(step), "step %d" % step, compare_tensors=(step in (0, 999)))
+        total += st.r
+    assert abs(st.tau - ost["tau"]) <= 1e-4 * ost["tau"]
+    assert st.tau == pytest.approx(total, rel=1e-12)
+    assert st.lr == pytest.approx(0.001)            # tau ~ 6400 has passed both boundaries (2000, 4000)
+    print("tau device %.9f oracle %.9f rel %.3g" % (st.tau, ost["tau"], abs(st.tau - ost["tau"]) / ost["tau"]))
+    pair.close()
+
+
 def test_transformer_base_heavy_tails_full_size():
     wl = synthetic.workload("transformer_base")
     src = synthetic.GradientSource(wl, device=DEV)
@@ -98,6 +117,24 @@ def test_decoder_24l_bf16_full_size():
     sample = [0, 1, 2, 3, 150, 291]
     for step, k in enumerate((0.1, 10.0)):
         st, _ = pair.step_streamed(src.fill(step, k=k), "k=%g" % k, sample_tensors=sample)
+    pair.close()
+
+
+@pytest.mark.skipif(os.environ.get("ADASCALE_FULL_TRAJECTORY") != "1",
+                    reason="about half an hour of copies and oracle time: set ADASCALE_FULL_TRAJECTORY=1")
+def test_decoder_24l_drifting_noise_200_steps_full_size():
+    """All 200 iterations of the drifting-noise workload at the full 354.8M parameters, S = 32, bf16."""
+    wl = synthetic.workload("decoder_24l")
+    src = synthetic.GradientSource(wl, device=DEV)
+    pair = _pair(wl, src)
+    rs = []
+    for step in range(200):
+        sample = [0, 2, 150, 291] if step in (0, 199) else []
+        st, ost = pair.step_streamed(src.fill(step), "step %d" % step, sample_tensors=sample)
+        rs.append(st.r)
+    assert rs[0] < 1.1 and rs[-1] > 10.0
+    assert abs(st.tau - ost["tau"]) <= 1e-5 * ost["tau"]
+    print("r first %.6f last %.6f tau device %.9f oracle %.9f" % (rs[0], rs[-1], st.tau, ost["tau"]))
     pair.close()
 
 
