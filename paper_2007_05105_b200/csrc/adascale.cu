@@ -479,6 +479,31 @@ template <int CPT> struct Cols<ADASCALE_BF16, CPT> {
     }
 };
 
+// The mean gradient is read again by the update kernel right after the reduce kernel ends and
+// overwritten by the next iteration: stored with the evict-last L2 priority it survives the
+// stream of gradient rows (which are evict-first) and mostly never travels to DRAM and back.
+__device__ __forceinline__ u64 l2_keep_policy()
+{
+    u64 p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+
+template <int CPT>
+__device__ __forceinline__ void store_cols_keep(float *g, const float *m, u64 policy)
+{
+    if constexpr (CPT == 2) {
+        asm volatile("st.global.L2::cache_hint.v2.f32 [%0], {%1, %2}, %3;" ::"l"(g), "f"(m[0]), "f"(m[1]), "l"(policy)
+                     : "memory");
+    } else {
+#pragma unroll
+        for (int k = 0; k < CPT; k += 4)
+            asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(g + k), "f"(m[k]),
+                         "f"(m[k + 1]), "f"(m[k + 2]), "f"(m[k + 3]), "l"(policy)
+                         : "memory");
+    }
+}
+
 template <int CPT>
 __device__ __forceinline__ void store_cols(float *g, const float *m)
 {
@@ -627,6 +652,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
             eta = eta_shared;
         }
         constexpr int NP = CPT / 2;
+        const u64 keep = l2_keep_policy();
         f2 c[NP], s1[NP], s2[NP], p1[NP];  // per-column state as packed pairs
         const long long G = gridDim.x;
         TileDesc d0, d1 = {};  // descriptor one tile ahead, as above
@@ -764,7 +790,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                             for (int j = 0; j < CPT; ++j) { vt[j] = vr[j]; wt[j] = wr[j]; }
                         }
                     } else {
-                        store_cols<CPT>(a.gbar + d0.goff + tid * CPT, m);
+                        store_cols_keep<CPT>(a.gbar + d0.goff + tid * CPT, m, keep);
                     }
                     accD += (double)dacc;
                     accN += (double)nacc;
