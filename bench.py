@@ -310,6 +310,29 @@ def run_ours(args, wl):
     torch.cuda.synchronize(dev)
     t_reduce = sum(a.elapsed_time(b) for a, b, c in ev) / ksteps
     t_update = sum(b.elapsed_time(c) for a, b, c in ev) / ksteps
+    # the same kernels launched back to back on their own (no neighbour's dirty lines to write back)
+    iso = {}
+    if not fused:
+        for name, call in (("reduce", lambda: ada.reduce(gp, sched)), ("update", lambda: ada.update(wp, vp))):
+            i0, i1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            for _ in range(3):
+                call()
+            i0.record(stream)
+            for _ in range(ksteps):
+                call()
+            i1.record(stream)
+            torch.cuda.synchronize(dev)
+            iso[name + "_us"] = i0.elapsed_time(i1) / ksteps * 1e3
+    # small working sets: also the warm figure (no L2 flush, steps back to back)
+    warm_ms = None
+    if flush is not None:
+        w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        w0.record(stream)
+        for _ in range(steps):
+            ada.step(gp, wp, vp, sched)
+        w1.record(stream)
+        torch.cuda.synchronize(dev)
+        warm_ms = w0.elapsed_time(w1) / steps
     peak, peak_kind = measured_peak()
     reduce_gbs = reduce_b / (t_reduce * 1e-3) / 1e9
     update_gbs = update_b / (t_update * 1e-3) / 1e9 if not fused else 0.0
@@ -389,9 +412,13 @@ def run_ours(args, wl):
             "roofline": {"bound": "hbm", "kernel": "k_reduce (fused)" if fused else "k_reduce", "achieved": reduce_gbs, "peak": peak, "unit": "GB/s",
                          "frac": reduce_gbs / peak, "peak_kind": peak_kind + " copy bandwidth", "traffic": None if fused else NCU_TRAFFIC_BYTES.get(wl.name),
                          "bytes_per_launch": reduce_b, "us_per_launch": t_reduce * 1e3,
+                         "timing": "events around each launch inside the step sequence (reduce, update, reduce, ...)",
+                         "back_to_back_alone": iso,
                          "update_kernel": None if fused else
                          {"kernel": "k_update", "achieved": update_gbs, "frac": update_gbs / peak,
                           "bytes_per_launch": update_b, "us_per_launch": t_update * 1e3}},
+            "warm_l2": None if warm_ms is None else {"ms_per_step": warm_ms, "value": step_b / (warm_ms * 1e-3) / 1e9,
+                                                     "note": "no L2 flush, steps back to back"},
             "ceilings": ceilings, "clocks": clocks, "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": launches,
         }
         print(json.dumps(line), flush=True)

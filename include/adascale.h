@@ -135,7 +135,9 @@ adascale_status adascale_init(const adascale_config *cfg, adascale_ctx **out);
 /*
  * One iteration (Sec. 3.2, App. B.3, Eq. 2-3): reduce + update, two kernel launches on
  * `cuda_stream` (a cudaStream_t passed as void*, NULL = default stream).  Returns after
- * enqueueing; never synchronises.
+ * enqueueing.  It waits for the device in one case only: when the tiling has to be rebuilt
+ * (first call, a new S, a tensor whose 16-byte alignment changed) the tile descriptors are
+ * uploaded and the call waits for that upload.
  *   grads    host array [S * T] of device pointers; row i, tensor k at [i*T + k];
  *            element type cfg.grad_dtype; read only.
  *   params   host array [T] of device pointers, float32, updated in place.

@@ -867,9 +867,6 @@ __device__ __forceinline__ void update4(float4 &ww, float4 &vv, const float4 &gg
 __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const __grid_constant__ UpdateArgs a)
 {
     griddep_launch();
-    griddep_wait();  // eta_t and the mean gradient come from the reduce kernel just before
-    if (a.st->status & ADASCALE_STATUS_NONFINITE) return;
-    const float eta = (float)a.st->eta;
     const int tid = threadIdx.x, T = a.T;
     const long long n_tiles = a.n_tiles, G = gridDim.x;
     // descriptor two tiles ahead, the tensor's pointers one tile ahead (see the reduce kernel)
@@ -883,6 +880,17 @@ __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const _
         fl_n = a.wflags[d1.tensor];
     }
     if ((long long)blockIdx.x + G < n_tiles) d2 = a.tiles[blockIdx.x + G];
+    // w and v of the first tile do not depend on the reduce kernel: they are requested while it
+    // still drains; eta_t and the mean gradient are read only after the wait
+    float4 w_first = make_float4(0.f, 0.f, 0.f, 0.f), v_first = w_first;
+    const bool first_fast = (long long)blockIdx.x < n_tiles && (fl_n & 1u) && d1.len == kUpdateTile;
+    if (first_fast) {
+        w_first = ((const float4 *)(wp_n + d1.first))[tid];
+        v_first = ((const float4 *)(vp_n + d1.first))[tid];
+    }
+    griddep_wait();
+    if (a.st->status & ADASCALE_STATUS_NONFINITE) return;
+    const float eta = (float)a.st->eta;
     for (long long t = blockIdx.x; t < n_tiles; t += G) {
         d0 = d1; wp = wp_n; vp = vp_n; fl = fl_n;
         d1 = d2;
@@ -898,9 +906,10 @@ __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const _
         const float *g = a.gbar + d0.goff;
         const bool vec = (fl & 1u) != 0;
         if (vec && len == kUpdateTile) {
+            const bool have = first_fast && t == (long long)blockIdx.x;
             const float4 gg = ((const float4 *)g)[tid];
-            float4 ww = ((const float4 *)w)[tid];
-            float4 vv = ((const float4 *)v)[tid];
+            float4 ww = have ? w_first : ((const float4 *)w)[tid];
+            float4 vv = have ? v_first : ((const float4 *)v)[tid];
             update4(ww, vv, gg, a.rho, a.lambda, eta);
             ((float4 *)v)[tid] = vv;
             ((float4 *)w)[tid] = ww;
