@@ -26,7 +26,8 @@ if ROOT not in sys.path:
 METRIC = "adascale_step gradient GB/s and % of B200 HBM peak; step latency (us)"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the reduce kernel, from the ncu
 # captures summarised under profiles/ (same kernel build); None where no capture exists
-NCU_TRAFFIC_BYTES = {"resnet18": 382.5e6, "resnet50": 875.4e6}
+NCU_TRAFFIC_BYTES = {"resnet18": 383.4e6, "resnet50": 855.7e6}
+NCU_TRAFFIC_BYTES_FUSED = {"resnet18": 510.7e6}
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 L2_BYTES = 126 * 1024 * 1024
@@ -410,7 +411,7 @@ def run_ours(args, wl):
                        else ("inputs larger than L2 (working set %d MB)" % (working_set >> 20)),
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "roofline": {"bound": "hbm", "kernel": "k_reduce (fused)" if fused else "k_reduce", "achieved": reduce_gbs, "peak": peak, "unit": "GB/s",
-                         "frac": reduce_gbs / peak, "peak_kind": peak_kind + " copy bandwidth", "traffic": None if fused else NCU_TRAFFIC_BYTES.get(wl.name),
+                         "frac": reduce_gbs / peak, "peak_kind": peak_kind + " copy bandwidth", "traffic": NCU_TRAFFIC_BYTES_FUSED.get(wl.name) if fused else NCU_TRAFFIC_BYTES.get(wl.name),
                          "bytes_per_launch": reduce_b, "us_per_launch": t_reduce * 1e3,
                          "timing": "events around each launch inside the step sequence (reduce, update, reduce, ...)",
                          "back_to_back_alone": iso,
