@@ -44,7 +44,7 @@ def _params(numels, gen, misalign=0):
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
-@pytest.mark.parametrize("S", [1, 2, 3, 4, 5, 7, 8, 9, 16, 17, 32, 33, 40])
+@pytest.mark.parametrize("S", [1, 2, 3, 4, 5, 7, 8, 9, 16, 17, 32, 33, 40, 128])
 def test_ragged_tensor_list(S, dtype):
     gen = _gen(1000 + S)
     name = "bf16" if dtype == torch.bfloat16 else "f32"
@@ -402,3 +402,53 @@ def test_fused_mode_call_rules():
             call()
         assert e.value.status == B.ERR_STATE
     ada.close()
+
+
+def test_one_tensor_with_more_than_2_31_elements():
+    """64-bit offsets: a single bf16 tensor of 2^31 + 4101 elements, S = 2, rows x and -x.
+
+    Too large for the CPU oracle in test time; the expected values follow from the construction:
+    gbar = 0 exactly, so N = 0, D = 2 sum x^2 (torch fp64 reduction, an independent routine),
+    v <- rho v + lambda w and w <- w - eta v.
+    """
+    n = (1 << 31) + 4101
+    gen = _gen(4000)
+    x = torch.empty(n, device=DEV, dtype=torch.bfloat16)
+    for lo in range(0, n, 1 << 28):
+        hi = min(n, lo + (1 << 28))
+        x[lo:hi] = torch.empty(hi - lo, device=DEV).normal_(0, 1, generator=gen).to(torch.bfloat16)
+    neg = -x
+    w = torch.full((n,), 2.0, device=DEV)
+    v = torch.full((n,), 0.5, device=DEV)
+    ada = B.AdaScale([n], 2, "bf16", momentum=0.5, weight_decay=0.25, theta=0.0)
+    ada.step([[x], [neg]], [w], [v], B.make_schedule("const", eta0=0.125))
+    st = ada.get_gain_tau(True)
+    sq = 0.0
+    for lo in range(0, n, 1 << 28):
+        sq += float(x[lo:min(n, lo + (1 << 28))].double().pow(2).sum())
+    assert st.gbar_sqnorm == 0.0
+    assert st.dev_sqsum == pytest.approx(2.0 * sq, rel=1e-6)
+    # sigma^2 = D, mu^2 = -D/2 -> clamped to 0 -> r = S = 2, eta = 0.25; v = 0.25 + 0.5 = 0.75, w = 2 - 0.1875
+    assert st.r == pytest.approx(2.0, rel=1e-12) and st.eta == pytest.approx(0.25, rel=1e-12)
+    gbar = ada.mean_grad_tensors()[0]
+    for sl in (slice(0, 4096), slice((1 << 31) - 2048, (1 << 31) + 2048), slice(n - 4101, n)):
+        assert bool((gbar[sl] == 0).all())
+        assert bool((v[sl] == 0.75).all()) and bool((w[sl] == 2.0 - 0.25 * 0.75).all())
+    assert float(v.min()) == 0.75 and float(v.max()) == 0.75
+    assert float(w.min()) == 1.8125 and float(w.max()) == 1.8125
+    ada.close()
+
+
+def test_scale_of_one_thousand_rows():
+    """S = 1000: many row chunks per tile, and the paper's theta rule gives 0 (no averaging)."""
+    gen = _gen(4100)
+    numels = [3000, 7]
+    # r is several hundred here, so the base rate is small: eta_t = r_t * lr stays of order 0.01-0.1
+    pair = H.Pair(numels, 1000, "f32", momentum=0.9, lr={"kind": "const", "eta0": 1e-4})
+    assert pair.orc.theta == 0.0
+    w, v = _params(numels, gen)
+    pair.attach(w, v)
+    for step in range(2):
+        st, _ = pair.step(_make_rows(numels, 1000, torch.float32, gen, k=30.0), "S=1000 step %d" % step)
+    assert 1.0 <= st.r <= 1000.0
+    pair.close()
