@@ -7,7 +7,8 @@ import sys
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 SOURCES = [os.path.join(_HERE, "csrc", "adascale.cu")]
-HEADER = os.path.join(os.path.dirname(_HERE), "include", "adascale.h")
+HEADERS = [os.path.join(os.path.dirname(_HERE), "include", "adascale.h"),
+           os.path.join(_HERE, "csrc", "adascale_kernels.cuh")]
 LIB = os.path.join(_HERE, "libadascale_b200.so")
 
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
@@ -25,7 +26,7 @@ def stale() -> bool:
     if not os.path.exists(LIB):
         return True
     built = os.path.getmtime(LIB)
-    return any(os.path.getmtime(p) > built for p in SOURCES + [HEADER])
+    return any(os.path.getmtime(p) > built for p in SOURCES + HEADERS)
 
 
 def build(force: bool = False, verbose: bool = False) -> str:

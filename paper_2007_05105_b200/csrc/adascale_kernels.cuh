@@ -1,0 +1,968 @@
+#pragma once
+// AdaScale SGD gain-ratio step for sm_100a: device code (the host glue is in adascale.cu).
+//
+// Two kernels make up one iteration (paper: Sec. 3.2, App. B.3, Eq. 2-3):
+//   reduce  - streams the S x P gradient matrix once through shared memory (bulk asynchronous
+//             copies completed on mbarriers, a producer warp and eight consumer warps), writes
+//             the mean gradient and one pair (sum of squared deviations, squared norm of the
+//             mean) per block; the block that finishes last adds the pairs in index order and
+//             runs the scalar part (estimates, clamps, moving averages, r_t, eta_t, tau_{t+1}).
+//   update  - v <- rho v + (gbar + lambda w), w <- w - eta_t v, reading eta_t from the device.
+// Three trivial streaming kernels calibrate the bandwidth ceiling.
+// The path is bound by HBM bandwidth; there is no contraction, hence no tensor-core work.
+//
+// Work distribution: every tensor is cut into tiles; tile t belongs to block t mod gridDim.
+// All blocks therefore advance through each gradient row as one front, which keeps DRAM
+// pages hot, and the split does not depend on how the hardware schedules blocks, so the
+// fixed-order sums are reproducible from run to run.
+#include "../../include/adascale.h"
+
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <string>
+#include <vector>
+
+namespace {
+
+constexpr int kThreads = 256;             // consumer threads of the reduce kernel, all threads of the update kernel
+constexpr int kWarps = kThreads / 32;
+constexpr int kStagedThreads = kThreads + 32;  // + 1 producer warp
+constexpr int kStagedWarps = kStagedThreads / 32;
+constexpr int kStages = 3;                // shared-memory stages per block
+constexpr int kMaxRowsPerStage = 16;      // rows of one stage; larger S goes through in row chunks
+constexpr int kStageBytes = 32 * 1024;    // upper bound of one stage
+constexpr int kReduceBlocksPerSM = 2;
+constexpr int kUpdateBlocksPerSM = 8;
+constexpr int kScalarTile = 2048;         // elements per tile on the unaligned / ragged-tail path
+constexpr int kUpdateTile = 1024;         // elements per tile of the update kernel: one 128-bit access per thread
+constexpr int kGbarAlign = 64;            // every tensor's mean gradient starts on a 256-byte boundary
+constexpr int kRing = 4;                  // pinned staging slots for pointer-table uploads
+constexpr int kMaxS = 4096;
+constexpr unsigned kSpinLimit = 1u << 22; // bounded waits: give up, flag, leave
+
+typedef unsigned long long u64;
+
+// Scalar state kept on the device between iterations.
+struct DevState {
+    double tau;    // scale-invariant iteration tau_t
+    double avg_a;  // sigma_bar^2 (ratio estimator: m1)
+    double avg_b;  // mu_bar^2    (ratio estimator: m2)
+    long long n;   // samples absorbed by the averages
+    long long t;   // iterations applied
+    long long skipped;
+    double r, eta, lr;
+    double sigma2_raw, mu2_raw;
+    double N, D;
+    unsigned status;
+    unsigned fault;  // sticky: a bounded device-side wait gave up
+};
+
+struct ScalarCfg {
+    double eps, theta;  // theta already resolved on the host (the paper's rule follows S)
+    unsigned flags;
+    int S;
+};
+
+struct Sched {
+    int kind, n;
+    double eta0, decay, t_s1;
+    double w[ADASCALE_MAX_MILESTONES];
+};
+
+// One tile of work: `len` elements of tensor `tensor` starting at element `first`; `goff` is
+// where the tile's mean gradient lives in the library's workspace.  Tile t belongs to block
+// t mod gridDim.  The descriptors hold no pointers, so they change only with the tiling.
+struct __align__(16) TileDesc {
+    long long first;
+    long long goff;
+    int tensor;
+    int len;
+    int pad[2];
+};
+
+// Reduce kernel: a tensor whose S row pointers are 16-byte aligned contributes staged tiles of
+// kThreads * CPT columns for its first numel & ~7 elements and one scalar tile for the ragged
+// rest; any other tensor contributes only scalar tiles of kScalarTile elements.
+struct ReduceArgs {
+    const u64 *gptr;          // [S * T] row pointers
+    const TileDesc *tiles;    // staged tiles
+    const TileDesc *stiles;   // scalar-path tiles
+    long long n_tiles, n_stiles;
+    float *gbar;
+    const u64 *wv;            // fused mode only: [2 * T] parameters then momentum
+    const unsigned *wflags;   // fused mode only: [T] bit0: both pointers 16-byte aligned
+    float rho, lambda;        // fused mode only
+    double2 *partials;
+    unsigned *ticket;
+    DevState *st;
+    int S, T;
+    float invS, fS;
+    ScalarCfg sc;
+    Sched sched;
+};
+
+struct UpdateArgs {
+    const u64 *wv;            // [2 * T]: parameters then momentum
+    const unsigned *wflags;   // [T] bit0: both pointers 16-byte aligned
+    const TileDesc *tiles;    // tiles of kUpdateTile elements
+    long long n_tiles;
+    const float *gbar;
+    const DevState *st;
+    int T;
+    float rho, lambda;
+};
+
+// Streaming 128-bit load (read once, evict first): used by the bandwidth probes.
+__device__ __forceinline__ uint4 ld_stream16(const void *p)
+{
+    uint4 r;
+    asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p));
+    return r;
+}
+
+// Element types of the gradient rows.  A bf16 is the upper half of an fp32, so widening is a
+// shift and exact.
+template <int DT> struct Elem;
+template <> struct Elem<ADASCALE_F32> {
+    static constexpr int kBytes = 4;
+    static __device__ __forceinline__ float load1(const void *p) { return __ldcs((const float *)p); }
+};
+template <> struct Elem<ADASCALE_BF16> {
+    static constexpr int kBytes = 2;
+    static __device__ __forceinline__ float load1(const void *p)
+    {
+        return __uint_as_float((unsigned)__ldcs((const unsigned short *)p) << 16);
+    }
+};
+
+// d = x - c, blocked first moment, running second moment, for V columns of one row.
+template <int V>
+__device__ __forceinline__ void accumulate_row(const float *x, const float *c, float *p1, float *s2)
+{
+#pragma unroll
+    for (int k = 0; k < V; ++k) {
+        const float d = x[k] - c[k];
+        p1[k] += d;
+        s2[k] = fmaf(d, d, s2[k]);
+    }
+}
+
+// One column, any alignment, any S: plain two-pass with a residual correction of the mean.
+// Row pointers come straight from the device table.
+template <int DT>
+__device__ __forceinline__ void column_scalar(const u64 *gptr, int T, int tensor, size_t boff, int S,
+                                                     float fS, float *gb, float &dsum, float &nsum)
+{
+    float sum = 0.f;
+    for (int i = 0; i < S; ++i) sum += Elem<DT>::load1((const char *)gptr[(size_t)i * T + tensor] + boff);
+    const float m0 = sum / fS;
+    float e = 0.f, qq = 0.f;
+    for (int i = 0; i < S; ++i) {
+        const float d = Elem<DT>::load1((const char *)gptr[(size_t)i * T + tensor] + boff) - m0;
+        e += d;
+        qq = fmaf(d, d, qq);
+    }
+    const float corr = e / fS;
+    const float m = m0 + corr;
+    *gb = m;
+    dsum = fmaf(-corr, e, qq);
+    nsum = m * m;
+}
+
+__device__ __forceinline__ double warp_sum(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Fixed-shape block sum of two doubles over NW warps; result valid in thread 0.
+template <int NW = kWarps>
+__device__ __forceinline__ void block_sum2(double &a, double &b, double *sa, double *sb)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    a = warp_sum(a);
+    b = warp_sum(b);
+    __syncthreads();  // scratch may still be in use by a previous call
+    if (lane == 0) {
+        sa[warp] = a;
+        sb[warp] = b;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        a = lane < NW ? sa[lane] : 0.0;
+        b = lane < NW ? sb[lane] : 0.0;
+        a = warp_sum(a);
+        b = warp_sum(b);
+    }
+}
+
+// App. B.1
+__device__ double lr_eval(const Sched &s, double t)
+{
+    if (s.kind == ADASCALE_LR_EXP) return s.eta0 * pow(s.decay, t / s.t_s1);
+    if (s.kind == ADASCALE_LR_STEP) {
+        int passed = 0;
+        for (int i = 0; i < s.n; ++i) passed += (t > s.w[i]) ? 1 : 0;
+        return s.eta0 * pow(s.decay, (double)passed);
+    }
+    return s.eta0;
+}
+
+__device__ __forceinline__ double ema(double prev, double sample, double theta, long long n)
+{
+    // plain mean of the first samples until the exponential weight takes over (App. B.3)
+    double warm = 1.0 - 1.0 / (double)n;
+    double th = theta < warm ? theta : warm;
+    return th * prev + (1.0 - th) * sample;
+}
+
+// Scalar part of the iteration: one thread, fp64, no host involvement.
+__device__ void scalar_step(DevState *st, const ScalarCfg &c, const Sched &sched, double D, double N)
+{
+    st->D = D;
+    st->N = N;
+    if (!isfinite(D) || !isfinite(N)) {  // skip the iteration, leave every average and tau alone
+        st->status = ADASCALE_STATUS_NONFINITE;
+        st->skipped += 1;
+        st->eta = 0.0;
+        return;
+    }
+    st->status = 0;
+    const double S = (double)c.S;
+    const double tau = st->tau;
+    const double t_arg = (c.flags & ADASCALE_FLAG_CONT_TAU) ? tau : floor(tau);
+    double r;
+    if (c.S == 1) {  // App. A.2: unit gain at scale one
+        st->sigma2_raw = 0.0;
+        st->mu2_raw = N;
+        r = 1.0;
+    } else {
+        double a, b, r_prior;
+        const bool ratio = (c.flags & ADASCALE_FLAG_RATIO) != 0;
+        if (ratio) {
+            // Sec. 3.4: (1/S) sum_i ||g_i||^2 = D/S + N  and ||gbar||^2
+            a = D / S + N;
+            b = N;
+            st->sigma2_raw = a;
+            st->mu2_raw = b;
+            r_prior = st->n > 0 ? (st->avg_a + c.eps) / (st->avg_b + c.eps) : 1.0;
+        } else {
+            // App. B.3: sigma^2 = D/(S-1) equals 1/(S-1) sum||g_i||^2 - S/(S-1)||gbar||^2
+            double sigma2 = D / (S - 1.0);
+            double mu2 = N - sigma2 / S;
+            st->sigma2_raw = sigma2;
+            st->mu2_raw = mu2;
+            a = sigma2 > c.eps ? sigma2 : c.eps;
+            b = mu2 > 0.0 ? mu2 : 0.0;
+            r_prior = st->n > 0 ? (st->avg_a + st->avg_b) / (st->avg_a / S + st->avg_b) : 1.0;
+        }
+        const long long n = st->n + 1;
+        const double na = ema(st->avg_a, a, c.theta, n);
+        const double nb = ema(st->avg_b, b, c.theta, n);
+        st->n = n;
+        st->avg_a = na;
+        st->avg_b = nb;
+        if (c.flags & ADASCALE_FLAG_LAGGED)
+            r = r_prior;
+        else
+            r = ratio ? (na + c.eps) / (nb + c.eps) : (na + nb) / (na / S + nb);  // Eq. 3
+    }
+    const double lr = lr_eval(sched, t_arg);
+    st->r = r;
+    st->lr = lr;
+    st->eta = r * lr;     // Sec. 3.2
+    st->tau = tau + r;
+    st->t += 1;
+}
+
+// Persistent grid: every block walks its own segments and keeps two fp64 accumulators per
+// thread for the whole launch, so there is one block reduction and one partial pair per block.
+// Lagged estimate (App. B.3: r_t from the averages of prior iterations only, r_0 = 1): the
+// learning rate of the coming iteration is known before its gradients are read.  Same
+// expressions as in scalar_step, so both give the identical value.
+__device__ double lagged_eta(const DevState *st, const ScalarCfg &c, const Sched &sched)
+{
+    const double S = (double)c.S;
+    double r = 1.0;
+    if (c.S > 1 && st->n > 0)
+        r = (c.flags & ADASCALE_FLAG_RATIO) ? (st->avg_a + c.eps) / (st->avg_b + c.eps)
+                                            : (st->avg_a + st->avg_b) / (st->avg_a / S + st->avg_b);
+    const double tau = st->tau;
+    const double t_arg = (c.flags & ADASCALE_FLAG_CONT_TAU) ? tau : floor(tau);
+    return r * lr_eval(sched, t_arg);
+}
+
+// Programmatic dependent launch: a kernel lets its successor in the stream be scheduled
+// early, and waits for its predecessor (completion and visibility of its writes) only where
+// it first depends on it.  Both are no-ops for a launch without the attribute.
+__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+__device__ __forceinline__ unsigned smem_u32(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(u64 *bar, unsigned count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(u64 *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(u64 *bar, unsigned bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Returns false if the phase did not complete within the spin limit.
+__device__ __forceinline__ bool mbar_wait(u64 *bar, unsigned parity)
+{
+    const unsigned addr = smem_u32(bar);
+    for (unsigned spin = 0; spin < kSpinLimit; ++spin) {
+        unsigned done;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done)
+                     : "r"(addr), "r"(parity)
+                     : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+// global -> shared bulk copy; bytes and both addresses are multiples of 16.  The rows are read
+// once: evict-first in L2 leaves the cache to the mean gradient that the update reads next.
+__device__ __forceinline__ void bulk_load(void *dst, const void *src, unsigned bytes, u64 *bar, u64 policy)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
+                 : "memory");
+}
+
+// ---- packed fp32 pairs -------------------------------------------------------------------
+// sm_100 adds, subtracts and multiply-adds two fp32 values with one instruction (f32x2).  The
+// consumer loop of the reduce kernel keeps its per-column state in such pairs: same IEEE
+// operations in the same order as scalar code, half the instruction issue.
+typedef unsigned long long f2;
+
+__device__ __forceinline__ f2 pack2(float lo, float hi)
+{
+    f2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f2 v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f2 add2(f2 a, f2 b)
+{
+    f2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f2 sub2(f2 a, f2 b)
+{
+    f2 r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f2 fma2(f2 a, f2 b, f2 c)
+{
+    f2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+// a bf16 pair in one 32-bit word -> two fp32 (widening is a shift / a mask, exact)
+__device__ __forceinline__ f2 widen2(unsigned u)
+{
+    f2 r;
+    asm("{\n\t.reg .b32 lo, hi;\n\tshl.b32 lo, %1, 16;\n\tand.b32 hi, %1, 0xffff0000;\n\tmov.b64 %0, {lo, hi};\n\t}"
+        : "=l"(r)
+        : "r"(u));
+    return r;
+}
+
+// CPT columns of one staged row, from shared memory (32-bit shared address plus a
+// compile-time byte offset), as CPT/2 packed pairs.
+template <int DT, int CPT> struct PairLoad;
+template <int CPT> struct PairLoad<ADASCALE_F32, CPT> {
+    template <int OFF>
+    static __device__ __forceinline__ void load(unsigned addr, f2 *x)
+    {
+        if constexpr (CPT == 2) {
+            asm volatile("ld.shared.b64 %0, [%1+%2];" : "=l"(x[0]) : "r"(addr), "n"(OFF));
+        } else {
+#pragma unroll
+            for (int k = 0; k < CPT / 4; ++k)
+                asm volatile("ld.shared.v2.b64 {%0, %1}, [%2+%3];"
+                             : "=l"(x[2 * k]), "=l"(x[2 * k + 1])
+                             : "r"(addr + 16 * k), "n"(OFF));
+        }
+    }
+};
+template <int CPT> struct PairLoad<ADASCALE_BF16, CPT> {
+    template <int OFF>
+    static __device__ __forceinline__ void load(unsigned addr, f2 *x)
+    {
+        if constexpr (CPT == 4) {
+            unsigned u0, u1;
+            asm volatile("ld.shared.v2.b32 {%0, %1}, [%2+%3];" : "=r"(u0), "=r"(u1) : "r"(addr), "n"(OFF));
+            x[0] = widen2(u0);
+            x[1] = widen2(u1);
+        } else {
+            unsigned u0, u1, u2, u3;
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4+%5];"
+                         : "=r"(u0), "=r"(u1), "=r"(u2), "=r"(u3)
+                         : "r"(addr), "n"(OFF));
+            x[0] = widen2(u0);
+            x[1] = widen2(u1);
+            x[2] = widen2(u2);
+            x[3] = widen2(u3);
+        }
+    }
+};
+
+// One staged row into the running sums: d = x - c, p1 += d, s2 += d * d.
+template <int DT, int CPT, int OFF>
+__device__ __forceinline__ void consume_row(unsigned addr, const f2 *c, f2 *p1, f2 *s2)
+{
+    f2 x[CPT / 2];
+    PairLoad<DT, CPT>::template load<OFF>(addr, x);
+#pragma unroll
+    for (int j = 0; j < CPT / 2; ++j) {
+        const f2 d = sub2(x[j], c[j]);
+        p1[j] = add2(p1[j], d);
+        s2[j] = fma2(d, d, s2[j]);
+    }
+}
+
+template <int DT, int CPT> struct Cols;
+template <int CPT> struct Cols<ADASCALE_F32, CPT> {
+    static __device__ __forceinline__ void load(const char *p, float *x)
+    {
+        if constexpr (CPT == 1) {
+            x[0] = *(const float *)p;
+        } else if constexpr (CPT == 2) {
+            const float2 t = *(const float2 *)p;
+            x[0] = t.x; x[1] = t.y;
+        } else {
+#pragma unroll
+            for (int k = 0; k < CPT; k += 4) {
+                const float4 t = *(const float4 *)(p + 4 * k);
+                x[k] = t.x; x[k + 1] = t.y; x[k + 2] = t.z; x[k + 3] = t.w;
+            }
+        }
+    }
+};
+template <int CPT> struct Cols<ADASCALE_BF16, CPT> {
+    static __device__ __forceinline__ void widen(unsigned u, float *x)
+    {
+        x[0] = __uint_as_float(u << 16);
+        x[1] = __uint_as_float(u & 0xffff0000u);
+    }
+    static __device__ __forceinline__ void load(const char *p, float *x)
+    {
+        if constexpr (CPT == 2) {
+            widen(*(const unsigned *)p, x);
+        } else if constexpr (CPT == 4) {
+            const uint2 t = *(const uint2 *)p;
+            widen(t.x, x); widen(t.y, x + 2);
+        } else {
+            const uint4 t = *(const uint4 *)p;
+            widen(t.x, x); widen(t.y, x + 2); widen(t.z, x + 4); widen(t.w, x + 6);
+        }
+    }
+};
+
+// The mean gradient is read again by the update kernel right after the reduce kernel ends and
+// overwritten by the next iteration: stored with the evict-last L2 priority it survives the
+// stream of gradient rows (which are evict-first) and mostly never travels to DRAM and back.
+__device__ __forceinline__ u64 l2_keep_policy()
+{
+    u64 p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+
+template <int CPT>
+__device__ __forceinline__ void store_cols_keep(float *g, const float *m, u64 policy)
+{
+    if constexpr (CPT == 2) {
+        asm volatile("st.global.L2::cache_hint.v2.f32 [%0], {%1, %2}, %3;" ::"l"(g), "f"(m[0]), "f"(m[1]), "l"(policy)
+                     : "memory");
+    } else {
+#pragma unroll
+        for (int k = 0; k < CPT; k += 4)
+            asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(g + k), "f"(m[k]),
+                         "f"(m[k + 1]), "f"(m[k + 2]), "f"(m[k + 3]), "l"(policy)
+                         : "memory");
+    }
+}
+
+template <int CPT>
+__device__ __forceinline__ void store_cols(float *g, const float *m)
+{
+    if constexpr (CPT == 1) {
+        g[0] = m[0];
+    } else if constexpr (CPT == 2) {
+        *(float2 *)g = make_float2(m[0], m[1]);
+    } else {
+#pragma unroll
+        for (int k = 0; k < CPT; k += 4) *(float4 *)(g + k) = make_float4(m[k], m[k + 1], m[k + 2], m[k + 3]);
+    }
+}
+
+
+// ---------------------------------------------------------------------------------------
+// Reduce kernel.
+//
+// Per column the S values are shifted by a value c taken from the data:  d_i = g_i - c.
+// With s1 = sum d_i and s2 = sum d_i^2 the mean is c + s1/S and the summed squared
+// deviation is s2 - s1^2/S.  Because c is (close to) a sample, the subtraction loses a
+// factor of order S at worst, not the |mean|^2/sigma^2 that the raw formula of App. B.3
+// loses; identical rows give exactly zero; and each row is consumed as it is read.
+//   - c is the median of the first three rows (row 0 when S < 3): one outlier among them
+//     cannot become the shift, which keeps |s1|, and with it the rounding error of the
+//     mean, small under heavy-tailed noise.
+//   - s1 is summed in blocks of 8 rows (a fresh partial per block, then one add), so the
+//     long chain of roundings happens on small partial sums.
+//   - per-column results enter fp64 accumulators; warp shuffles, a block tree and a
+//     fixed-order second stage do the rest in fp64.
+//
+// A producer warp streams tiles into shared memory with bulk asynchronous copies (one copy
+// per row, completion counted on an mbarrier); eight consumer warps read them back.  Memory
+// latency is covered by the stages in flight rather than by registers, and the consumers
+// issue no global loads or address arithmetic.  A work item is (tile, row chunk):
+// kThreads * CPT columns of up to kMaxRowsPerStage rows.  Row chunks let any S through: the
+// per-column sums carry over from one chunk of rows to the next and close after the last.
+// ---------------------------------------------------------------------------------------
+//
+// FUSED (lagged estimate only): eta_t is known when the kernel starts, so the same pass also
+// reads w and v, applies the update of Eq. 2 and writes them back; the mean gradient lives in
+// registers only and the update kernel is not launched: P * (S * b_g + 16) bytes per iteration
+// instead of P * (S * b_g + 24), one launch instead of two.
+template <int DT, int CPT, bool FUSED>
+__global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(const __grid_constant__ ReduceArgs a)
+{
+    extern __shared__ __align__(128) unsigned char stage_mem[];
+    __shared__ __align__(8) u64 full_bar[kStages], empty_bar[kStages];
+    __shared__ double sa[kStagedWarps], sb[kStagedWarps];
+    __shared__ bool is_last;
+    __shared__ int abort_flag;
+    __shared__ float eta_shared;
+
+    constexpr int E = Elem<DT>::kBytes;
+    constexpr int kTile = kThreads * CPT;  // columns per tile
+    constexpr int kRowBytes = kTile * E;   // one row of a stage
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const bool producer = warp == kStagedWarps - 1;
+    const int S = a.S, T = a.T;
+    const int rps = S < kMaxRowsPerStage ? S : kMaxRowsPerStage;  // rows per stage
+    const int n_chunks = (S + rps - 1) / rps;
+    const unsigned stage_bytes = (unsigned)rps * kRowBytes;
+    const long long n_tiles = a.n_tiles;
+
+    griddep_launch();
+    if (tid == 0) {
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(&full_bar[i], 1);
+            mbar_init(&empty_bar[i], kWarps);
+        }
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    double accD = 0.0, accN = 0.0;
+    unsigned item = 0;  // running count of staged work items, identical in every thread
+    bool timed_out = false;
+
+    if (producer) {
+        u64 policy;
+        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+        int last_use[kStages];
+#pragma unroll
+        for (int i = 0; i < kStages; ++i) last_use[i] = -1;
+        // Round-robin tiles make every block visit most tensors, so table misses must stay off
+        // the copy queue: the descriptor is fetched two tiles ahead and this lane's row pointer
+        // (row = lane when S <= 32) one tile ahead.
+        const long long G = gridDim.x;
+        TileDesc d0, d1 = {}, d2 = {};
+        const char *rowptr = nullptr, *rowptr_n = nullptr;
+        if ((long long)blockIdx.x < n_tiles) d1 = a.tiles[blockIdx.x];
+        if ((long long)blockIdx.x + G < n_tiles) d2 = a.tiles[blockIdx.x + G];
+        if ((long long)blockIdx.x < n_tiles && lane < S) rowptr_n = (const char *)a.gptr[(size_t)lane * T + d1.tensor];
+        for (long long t = blockIdx.x; t < n_tiles && !timed_out; t += G) {
+            d0 = d1;
+            rowptr = rowptr_n;
+            d1 = d2;
+            if (t + 2 * G < n_tiles) d2 = a.tiles[t + 2 * G];
+            if (t + G < n_tiles && d1.tensor != d0.tensor && lane < S)
+                rowptr_n = (const char *)a.gptr[(size_t)lane * T + d1.tensor];
+            const int k = d0.tensor;
+            const long long c0 = d0.first;
+            const int tc = d0.len;
+            for (int ch = 0; ch < n_chunks; ++ch, ++item) {
+                const int st = item % kStages;
+                const unsigned use = item / kStages;
+                if (!mbar_wait(&empty_bar[st], (use & 1u) ^ 1u)) { timed_out = true; break; }
+                const int r0 = ch * rps;
+                const int rows = S - r0 < rps ? S - r0 : rps;
+                if (lane == 0) mbar_expect_tx(&full_bar[st], (unsigned)rows * tc * E);
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < kStages; ++i)
+                    if (i == st) last_use[i] = (int)use;
+                unsigned char *dst = stage_mem + (size_t)st * stage_bytes;
+                if (r0 + rps <= 32) {
+                    // rows r0 .. r0+rows-1 live in lanes r0 .. : each lane copies its own row
+                    const int r = lane - r0;
+                    if (r >= 0 && r < rows)
+                        bulk_load(dst + (size_t)r * kRowBytes, rowptr + (size_t)c0 * E, (unsigned)tc * E, &full_bar[st], policy);
+                } else {
+                    for (int r = lane; r < rows; r += 32) {
+                        const char *src = (const char *)a.gptr[(size_t)(r0 + r) * T + k] + (size_t)c0 * E;
+                        bulk_load(dst + (size_t)r * kRowBytes, src, (unsigned)tc * E, &full_bar[st], policy);
+                    }
+                }
+            }
+        }
+        if (timed_out) atomicExch(&abort_flag, 1);
+        if (timed_out || *(volatile int *)&abort_flag) {
+            // leaving early: copies already issued must land before this block's shared memory is reused
+#pragma unroll
+            for (int i = 0; i < kStages; ++i)
+                if (last_use[i] >= 0) mbar_wait(&full_bar[i], (unsigned)last_use[i] & 1u);
+        }
+    } else {
+        // The producer above may already stream gradient rows while the previous kernel in the
+        // stream (the update that still reads the old mean gradient) drains; nothing may be
+        // written before it has finished.
+        griddep_wait();
+        float eta = 0.f;
+        if constexpr (FUSED) {
+            if (tid == 0) eta_shared = (float)lagged_eta(a.st, a.sc, a.sched);
+            asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");  // consumers only
+            eta = eta_shared;
+        }
+        constexpr int NP = CPT / 2;
+        const u64 keep = l2_keep_policy();
+        f2 c[NP], s1[NP], s2[NP], p1[NP];  // per-column state as packed pairs
+        const long long G = gridDim.x;
+        TileDesc d0, d1 = {};  // descriptor one tile ahead, as above
+        if ((long long)blockIdx.x < n_tiles) d1 = a.tiles[blockIdx.x];
+        // fused mode: the tile's parameter and momentum pointers, fetched one tile ahead as well
+        float *wp = nullptr, *vp = nullptr, *wp_n = nullptr, *vp_n = nullptr;
+        unsigned fl = 0, fl_n = 0;
+        if constexpr (FUSED) {
+            if ((long long)blockIdx.x < n_tiles) {
+                wp_n = (float *)a.wv[d1.tensor];
+                vp_n = (float *)a.wv[T + d1.tensor];
+                fl_n = a.wflags[d1.tensor];
+            }
+        }
+        const unsigned lane_base = smem_u32(stage_mem) + (unsigned)tid * CPT * E;
+        for (long long t = blockIdx.x; t < n_tiles && !timed_out; t += G) {
+            d0 = d1;
+            if (t + G < n_tiles) d1 = a.tiles[t + G];
+            const int tc = d0.len;
+            const bool active = tid * CPT < tc;
+            float wr[CPT], vr[CPT];  // fused mode: this thread's parameters and momentum, requested
+            float *wt = nullptr, *vt = nullptr;  // before the rows are consumed so they arrive meanwhile
+            bool vec_wv = false;
+            if constexpr (FUSED) {
+                wp = wp_n; vp = vp_n; fl = fl_n;
+                if (t + G < n_tiles && d1.tensor != d0.tensor) {
+                    wp_n = (float *)a.wv[d1.tensor];
+                    vp_n = (float *)a.wv[T + d1.tensor];
+                    fl_n = a.wflags[d1.tensor];
+                }
+                wt = wp + d0.first + tid * CPT;
+                vt = vp + d0.first + tid * CPT;
+                vec_wv = (fl & 1u) != 0;
+                if (active) {
+                    if (vec_wv) {
+                        Cols<ADASCALE_F32, CPT>::load((const char *)wt, wr);
+                        Cols<ADASCALE_F32, CPT>::load((const char *)vt, vr);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < CPT; ++j) { wr[j] = wt[j]; vr[j] = vt[j]; }
+                    }
+                }
+            }
+            for (int ch = 0; ch < n_chunks; ++ch, ++item) {
+                const int st = item % kStages;
+                const unsigned use = item / kStages;
+                if (!mbar_wait(&full_bar[st], use & 1u)) { timed_out = true; break; }
+                const int r0 = ch * rps;
+                const int rows = S - r0 < rps ? S - r0 : rps;
+                unsigned addr = lane_base + (unsigned)st * stage_bytes;
+                if (active) {
+                    if (ch == 0) {
+                        if (S >= 3) {  // shift = median of the first three rows
+                            f2 x0[NP], x1[NP], x2[NP];
+                            PairLoad<DT, CPT>::template load<0>(addr, x0);
+                            PairLoad<DT, CPT>::template load<kRowBytes>(addr, x1);
+                            PairLoad<DT, CPT>::template load<2 * kRowBytes>(addr, x2);
+#pragma unroll
+                            for (int j = 0; j < NP; ++j) {
+                                float a0, a1, b0, b1, e0, e1;
+                                unpack2(x0[j], a0, a1);
+                                unpack2(x1[j], b0, b1);
+                                unpack2(x2[j], e0, e1);
+                                const float m0 = fmaxf(fminf(a0, b0), fminf(fmaxf(a0, b0), e0));
+                                const float m1 = fmaxf(fminf(a1, b1), fminf(fmaxf(a1, b1), e1));
+                                c[j] = pack2(m0, m1);
+                            }
+                        } else {
+                            PairLoad<DT, CPT>::template load<0>(addr, c);
+                        }
+#pragma unroll
+                        for (int j = 0; j < NP; ++j) s1[j] = s2[j] = 0ull;  // +0.0f, +0.0f
+                    }
+                    int r = 0;
+                    for (; r + 8 <= rows; r += 8) {  // s1 in blocks of 8 rows
+#pragma unroll
+                        for (int j = 0; j < NP; ++j) p1[j] = 0ull;
+                        consume_row<DT, CPT, 0 * kRowBytes>(addr, c, p1, s2);
+                        consume_row<DT, CPT, 1 * kRowBytes>(addr, c, p1, s2);
+                        consume_row<DT, CPT, 2 * kRowBytes>(addr, c, p1, s2);
+                        consume_row<DT, CPT, 3 * kRowBytes>(addr, c, p1, s2);
+                        consume_row<DT, CPT, 4 * kRowBytes>(addr, c, p1, s2);
+                        consume_row<DT, CPT, 5 * kRowBytes>(addr, c, p1, s2);
+                        consume_row<DT, CPT, 6 * kRowBytes>(addr, c, p1, s2);
+                        consume_row<DT, CPT, 7 * kRowBytes>(addr, c, p1, s2);
+#pragma unroll
+                        for (int j = 0; j < NP; ++j) s1[j] = add2(s1[j], p1[j]);
+                        addr += 8 * kRowBytes;
+                    }
+                    if (r < rows) {
+#pragma unroll
+                        for (int j = 0; j < NP; ++j) p1[j] = 0ull;
+                        for (; r < rows; ++r) {
+                            consume_row<DT, CPT, 0>(addr, c, p1, s2);
+                            addr += kRowBytes;
+                        }
+#pragma unroll
+                        for (int j = 0; j < NP; ++j) s1[j] = add2(s1[j], p1[j]);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty_bar[st]);  // this warp is done with the stage
+                if (active && ch == n_chunks - 1) {
+                    float m[CPT];
+                    float dacc = 0.f, nacc = 0.f;
+#pragma unroll
+                    for (int j = 0; j < NP; ++j) {
+                        float cc[2], ss1[2], ss2[2];
+                        unpack2(c[j], cc[0], cc[1]);
+                        unpack2(s1[j], ss1[0], ss1[1]);
+                        unpack2(s2[j], ss2[0], ss2[1]);
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            // quotient s1/S: reciprocal multiply plus one residual correction (1/S is not
+                            // exact unless S is a power of two, and a biased 1/S would bias every column alike)
+                            float q = ss1[h] * a.invS;
+                            const float res = fmaf(-q, a.fS, ss1[h]);
+                            q = fmaf(res, a.invS, q);
+                            m[2 * j + h] = cc[h] + q;
+                            dacc += fmaf(-q, ss1[h], ss2[h]);
+                            nacc = fmaf(m[2 * j + h], m[2 * j + h], nacc);
+                        }
+                    }
+                    if constexpr (FUSED) {
+#pragma unroll
+                        for (int j = 0; j < CPT; ++j) {
+                            vr[j] = fmaf(a.rho, vr[j], fmaf(a.lambda, wr[j], m[j]));
+                            wr[j] = fmaf(-eta, vr[j], wr[j]);
+                        }
+                        if (vec_wv) {
+                            store_cols<CPT>(vt, vr);
+                            store_cols<CPT>(wt, wr);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < CPT; ++j) { vt[j] = vr[j]; wt[j] = wr[j]; }
+                        }
+                    } else {
+                        store_cols_keep<CPT>(a.gbar + d0.goff + tid * CPT, m, keep);
+                    }
+                    accD += (double)dacc;
+                    accN += (double)nacc;
+                }
+            }
+        }
+        // ragged tails (< 8 elements) and tensors that are not 16-byte aligned: plain loads
+        for (long long t = blockIdx.x; t < a.n_stiles; t += gridDim.x) {
+            const TileDesc d = a.stiles[t];
+            float *gb = a.gbar + d.goff;
+            for (int e = tid; e < d.len; e += kThreads) {
+                float dd, nn;
+                if constexpr (FUSED) {
+                    float m;
+                    column_scalar<DT>(a.gptr, T, d.tensor, ((size_t)d.first + e) * E, S, a.fS, &m, dd, nn);
+                    float *w = (float *)a.wv[d.tensor] + d.first + e;
+                    float *v = (float *)a.wv[T + d.tensor] + d.first + e;
+                    const float vn = fmaf(a.rho, *v, fmaf(a.lambda, *w, m));
+                    *v = vn;
+                    *w = fmaf(-eta, vn, *w);
+                } else {
+                    column_scalar<DT>(a.gptr, T, d.tensor, ((size_t)d.first + e) * E, S, a.fS, gb + e, dd, nn);
+                }
+                accD += (double)dd;
+                accN += (double)nn;
+            }
+        }
+        if (timed_out) atomicExch(&abort_flag, 1);
+    }
+
+    block_sum2<kStagedWarps>(accD, accN, sa, sb);
+    if (tid == 0) {
+        if (abort_flag) atomicOr(&a.st->fault, ADASCALE_STATUS_WAIT_TIMEOUT);
+        a.partials[blockIdx.x] = make_double2(accD, accN);
+        __threadfence();
+        const unsigned tk = atomicAdd(a.ticket, 1u);
+        is_last = (tk == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+
+    // Second stage, fixed order: thread j adds partials j, j+288, ... in index order, then the
+    // same block tree.  The result depends on the tiling only, not on how blocks were scheduled.
+    __threadfence();
+    double d = 0.0, n = 0.0;
+    for (int i = tid; i < (int)gridDim.x; i += kStagedThreads) {
+        const double2 p = __ldcg(&a.partials[i]);
+        d += p.x;
+        n += p.y;
+    }
+    block_sum2<kStagedWarps>(d, n, sa, sb);
+    if (tid == 0) {
+        scalar_step(a.st, a.sc, a.sched, d, n);
+        *a.ticket = 0u;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Update kernel (Eq. 2 with momentum): tiles of kUpdateTile elements, one 128-bit access per
+// array and thread, tiles dealt round-robin like in the reduce kernel.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void update4(float4 &ww, float4 &vv, const float4 &gg, float rho, float lambda, float eta)
+{
+    vv.x = fmaf(rho, vv.x, fmaf(lambda, ww.x, gg.x));
+    vv.y = fmaf(rho, vv.y, fmaf(lambda, ww.y, gg.y));
+    vv.z = fmaf(rho, vv.z, fmaf(lambda, ww.z, gg.z));
+    vv.w = fmaf(rho, vv.w, fmaf(lambda, ww.w, gg.w));
+    ww.x = fmaf(-eta, vv.x, ww.x);
+    ww.y = fmaf(-eta, vv.y, ww.y);
+    ww.z = fmaf(-eta, vv.z, ww.z);
+    ww.w = fmaf(-eta, vv.w, ww.w);
+}
+
+__global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const __grid_constant__ UpdateArgs a)
+{
+    griddep_launch();
+    const int tid = threadIdx.x, T = a.T;
+    const long long n_tiles = a.n_tiles, G = gridDim.x;
+    // descriptor two tiles ahead, the tensor's pointers one tile ahead (see the reduce kernel)
+    TileDesc d0, d1 = {}, d2 = {};
+    float *wp = nullptr, *vp = nullptr, *wp_n = nullptr, *vp_n = nullptr;
+    unsigned fl = 0, fl_n = 0;
+    if ((long long)blockIdx.x < n_tiles) {
+        d1 = a.tiles[blockIdx.x];
+        wp_n = (float *)a.wv[d1.tensor];
+        vp_n = (float *)a.wv[T + d1.tensor];
+        fl_n = a.wflags[d1.tensor];
+    }
+    if ((long long)blockIdx.x + G < n_tiles) d2 = a.tiles[blockIdx.x + G];
+    // w and v of the first tile do not depend on the reduce kernel: they are requested while it
+    // still drains; eta_t and the mean gradient are read only after the wait
+    float4 w_first = make_float4(0.f, 0.f, 0.f, 0.f), v_first = w_first;
+    const bool first_fast = (long long)blockIdx.x < n_tiles && (fl_n & 1u) && d1.len == kUpdateTile;
+    if (first_fast) {
+        w_first = ((const float4 *)(wp_n + d1.first))[tid];
+        v_first = ((const float4 *)(vp_n + d1.first))[tid];
+    }
+    griddep_wait();
+    if (a.st->status & ADASCALE_STATUS_NONFINITE) return;
+    const float eta = (float)a.st->eta;
+    for (long long t = blockIdx.x; t < n_tiles; t += G) {
+        d0 = d1; wp = wp_n; vp = vp_n; fl = fl_n;
+        d1 = d2;
+        if (t + 2 * G < n_tiles) d2 = a.tiles[t + 2 * G];
+        if (t + G < n_tiles && d1.tensor != d0.tensor) {
+            wp_n = (float *)a.wv[d1.tensor];
+            vp_n = (float *)a.wv[T + d1.tensor];
+            fl_n = a.wflags[d1.tensor];
+        }
+        const long long first = d0.first;
+        const int len = d0.len;
+        float *w = wp + first, *v = vp + first;
+        const float *g = a.gbar + d0.goff;
+        const bool vec = (fl & 1u) != 0;
+        if (vec && len == kUpdateTile) {
+            const bool have = first_fast && t == (long long)blockIdx.x;
+            const float4 gg = ((const float4 *)g)[tid];
+            float4 ww = have ? w_first : ((const float4 *)w)[tid];
+            float4 vv = have ? v_first : ((const float4 *)v)[tid];
+            update4(ww, vv, gg, a.rho, a.lambda, eta);
+            ((float4 *)v)[tid] = vv;
+            ((float4 *)w)[tid] = ww;
+        } else {
+            int done = 0;
+            if (vec) {
+                const int nv = len >> 2;
+                if (tid < nv) {
+                    const float4 gg = ((const float4 *)g)[tid];
+                    float4 ww = ((const float4 *)w)[tid];
+                    float4 vv = ((const float4 *)v)[tid];
+                    update4(ww, vv, gg, a.rho, a.lambda, eta);
+                    ((float4 *)v)[tid] = vv;
+                    ((float4 *)w)[tid] = ww;
+                }
+                done = nv << 2;
+            }
+            for (int e = done + tid; e < len; e += kThreads) {
+                const float vn = fmaf(a.rho, v[e], fmaf(a.lambda, w[e], g[e]));
+                v[e] = vn;
+                w[e] = fmaf(-eta, vn, w[e]);
+            }
+        }
+    }
+}
+
+// ---- bandwidth probes -------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads) k_probe_read(const uint4 *a, long long n, unsigned *sink)
+{
+    unsigned acc = 0;
+    for (long long i = (long long)blockIdx.x * kThreads + threadIdx.x; i < n; i += (long long)gridDim.x * kThreads) {
+        const uint4 q = ld_stream16(a + i);
+        acc ^= q.x ^ q.y ^ q.z ^ q.w;
+    }
+    if (acc == 0x9e3779b9u) *sink = acc;  // keeps the loads alive, practically never taken
+}
+__global__ void __launch_bounds__(kThreads) k_probe_copy(const uint4 *a, uint4 *b, long long n)
+{
+    for (long long i = (long long)blockIdx.x * kThreads + threadIdx.x; i < n; i += (long long)gridDim.x * kThreads)
+        b[i] = ld_stream16(a + i);
+}
+__global__ void __launch_bounds__(kThreads) k_probe_rmw(float4 *a, const float4 *b, long long n)
+{
+    for (long long i = (long long)blockIdx.x * kThreads + threadIdx.x; i < n; i += (long long)gridDim.x * kThreads) {
+        float4 x = a[i];
+        const float4 y = b[i];
+        x.x += y.x;
+        x.y += y.y;
+        x.z += y.z;
+        x.w += y.w;
+        a[i] = x;
+    }
+}
+
+}  // namespace
