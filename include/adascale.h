@@ -15,7 +15,8 @@
  *
  * Everything above runs in CUDA kernels; nothing is computed on the host and no call
  * except adascale_get_gain_tau(blocking), adascale_get_state, adascale_set_state,
- * adascale_step_host and adascale_destroy waits for the device.
+ * adascale_step_host and adascale_destroy waits for the device (one exception: the call that
+ * first sees a new tiling uploads it and waits for that upload, see adascale_step).
  *
  * Conventions
  *   - "device pointer" = address in the global memory of the context's GPU;
