@@ -378,7 +378,7 @@ def run_ours(args, wl):
         e_ms = (time.perf_counter() - t0) * 1e3 / esteps
         e_ms = max_over_ranks(e_ms, world, dev)
         e2e = {"value": world * step_b / (e_ms * 1e-3) / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": 128, "ms_per_step": e_ms, "steps": esteps,
+               "d2h_bytes_per_step": 112, "ms_per_step": e_ms, "steps": esteps,
                "api": "adascale_step_host (pinned host gradients -> device staging -> step -> stats to host)"}
         del host_rows
 
