@@ -62,6 +62,7 @@ struct DevState {
     unsigned status;
     unsigned fault;  // sticky: a bounded device-side wait gave up
 };
+static_assert(sizeof(DevState) == 112, "the snapshot copied to the host is 112 bytes");
 
 struct ScalarCfg {
     double eps, theta;  // theta already resolved on the host (the paper's rule follows S)
