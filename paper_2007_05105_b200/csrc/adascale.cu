@@ -408,19 +408,18 @@ bool valid_sched(const adascale_lr_schedule *s)
     return true;
 }
 
-// Layout of the reduce table in 8-byte words: [max_S * T row pointers]
-adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const adascale_lr_schedule *sched,
-                          cudaStream_t s, bool fused)
+// Validates the caller's gradient pointers, rebuilds the tiling if the tile width or a tensor's
+// alignment changed, and uploads the pointer table ([max_S * T] row pointers).  Skipped entirely
+// when the pointers are those of the previous call.
+adascale_status sync_reduce_table(adascale_ctx *ctx, const void *const *grads, cudaStream_t s)
 {
     const int S = ctx->S, T = ctx->T;
     const size_t esz = ctx->dtype == ADASCALE_BF16 ? 2 : 4;
-    const int max_blocks = ctx->sms * kReduceBlocksPerSM;
     const size_t n_ptrs = (size_t)S * T;
-    // The usual case, the same pointers as in the previous call: nothing to validate, build or upload.
-    const bool unchanged = ctx->tg.valid && ctx->tiled_cpt != 0 && ctx->last_grads.size() == n_ptrs &&
-                           std::memcmp(ctx->last_grads.data(), grads, n_ptrs * sizeof(void *)) == 0;
-    int cpt = ctx->tiled_cpt;
-    if (!unchanged) {
+    if (ctx->tg.valid && ctx->tiled_cpt != 0 && ctx->last_grads.size() == n_ptrs &&
+        std::memcmp(ctx->last_grads.data(), grads, n_ptrs * sizeof(void *)) == 0)
+        return ADASCALE_OK;
+
     std::vector<u64> fresh(ctx->tg.words, 0);
     std::vector<unsigned char> aligned((size_t)T, 1);
     for (int k = 0; k < T; ++k) {
@@ -434,7 +433,7 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
             fresh[(size_t)i * T + k] = p;
         }
     }
-    cpt = choose_cpt(ctx->dtype, S, ctx->numel.data(), aligned.data(), T, max_blocks);
+    const int cpt = choose_cpt(ctx->dtype, S, ctx->numel.data(), aligned.data(), T, ctx->sms * kReduceBlocksPerSM);
     if (cpt != ctx->tiled_cpt || aligned != ctx->tiled_aligned) {
         // the tiling follows the tile width (a function of S) and the alignment of the pointers
         cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
@@ -446,11 +445,10 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
         std::vector<TileDesc> tiles;
         long long n_staged = 0;
         build_reduce_tiles(ctx->numel.data(), ctx->goff.data(), aligned.data(), T, kThreads * cpt, tiles, n_staged);
-        if ((long long)tiles.size() > ctx->rtiles_cap) return ADASCALE_ERR_TOO_LARGE;  // cannot happen: sized for the worst case
+        if ((long long)tiles.size() > ctx->rtiles_cap) return ADASCALE_ERR_TOO_LARGE;  // sized for the worst case
         if (!tiles.empty()) {
-            // pageable source: the runtime stages it before the call returns
             CU(cudaMemcpyAsync(ctx->d_rtiles, tiles.data(), tiles.size() * sizeof(TileDesc), cudaMemcpyHostToDevice, s));
-            CU(cudaStreamSynchronize(s));
+            CU(cudaStreamSynchronize(s));  // `tiles` goes out of scope
         }
         ctx->n_tiles = n_staged;
         ctx->n_stiles = (long long)tiles.size() - n_staged;
@@ -460,7 +458,18 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
     adascale_status st = table_sync(ctx, ctx->tg, fresh, s);
     if (st != ADASCALE_OK) return st;
     ctx->last_grads.assign(grads, grads + n_ptrs);
-    }
+    return ADASCALE_OK;
+}
+
+adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const adascale_lr_schedule *sched,
+                          cudaStream_t s, bool fused)
+{
+    const int S = ctx->S, T = ctx->T;
+    const size_t esz = ctx->dtype == ADASCALE_BF16 ? 2 : 4;
+    const int max_blocks = ctx->sms * kReduceBlocksPerSM;
+    adascale_status st = sync_reduce_table(ctx, grads, s);
+    if (st != ADASCALE_OK) return st;
+    const int cpt = ctx->tiled_cpt;
     const long long n_tiles = ctx->n_tiles, n_stiles = ctx->n_stiles;
     if (n_tiles + n_stiles == 0) return ADASCALE_OK;  // nothing but empty tensors
 
