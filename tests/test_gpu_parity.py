@@ -452,3 +452,43 @@ def test_scale_of_one_thousand_rows():
         st, _ = pair.step(_make_rows(numels, 1000, torch.float32, gen, k=30.0), "S=1000 step %d" % step)
     assert 1.0 <= st.r <= 1000.0
     pair.close()
+
+
+def test_steps_replayed_from_a_cuda_graph_match_eager_steps():
+    """adascale_step only enqueues, so once its tables are on the device it can be captured."""
+    gen = _gen(4200)
+    numels = [50000, 4097, 64]
+    rows = _make_rows(numels, 8, torch.float32, gen)
+    other = _make_rows(numels, 8, torch.float32, gen)
+    sched = B.make_schedule("exp", eta0=0.05, d=0.5, T_S1=20.0)
+
+    def fresh():
+        w, v = _params(numels, _gen(4201))
+        return B.AdaScale(numels, 8, momentum=0.9, weight_decay=1e-4), w, v
+
+    eager, we, ve = fresh()
+    for _ in range(4):
+        eager.step(rows, we, ve, sched)
+    ref = eager.get_gain_tau(True).as_dict()
+
+    ada, w, v = fresh()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        ada.step(rows, w, v, sched, stream=side.cuda_stream)       # step 1, eager: uploads tables and tiling
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            ada.step(rows, w, v, sched, stream=side.cuda_stream)   # captured once ...
+            with pytest.raises(B.AdaScaleError) as e:              # ... new pointers are refused, nothing enqueued
+                ada.step(other, w, v, sched, stream=side.cuda_stream)
+            assert e.value.status == B.ERR_STATE
+        for _ in range(3):                                          # ... replayed as steps 2, 3, 4
+            graph.replay()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    got = ada.get_gain_tau(True).as_dict()
+    assert got == ref
+    for a, b in zip(w + v, we + ve):
+        assert torch.equal(a, b)
+    eager.close()
+    ada.close()
