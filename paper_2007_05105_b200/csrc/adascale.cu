@@ -228,7 +228,7 @@ double resolve_theta(const adascale_ctx *c)
 
 // ---- tiling of the reduce kernel ---------------------------------------------------------
 
-int rows_per_stage(int S) { return S < kMaxRowsPerStage ? S : kMaxRowsPerStage; }
+int rows_per_stage(int dtype, int S) { return S < max_rows_per_stage(dtype) ? S : max_rows_per_stage(dtype); }
 
 long long staged_tiles(const long long *numel, const unsigned char *aligned, int T, int tile_cols)
 {
@@ -245,7 +245,7 @@ int choose_cpt(int dtype, int S, const long long *numel, const unsigned char *al
 {
     const int esz = dtype == ADASCALE_BF16 ? 2 : 4;
     int bpt = dtype == ADASCALE_BF16 ? 16 : 32;
-    while (bpt > 8 && rows_per_stage(S) * kThreads * bpt > kStageBytes) bpt >>= 1;
+    while (bpt > 8 && rows_per_stage(dtype, S) * kThreads * bpt > kStageBytes) bpt >>= 1;
     while (bpt > 8 && staged_tiles(numel, aligned, T, kThreads * bpt / esz) < 4LL * n_blocks) bpt >>= 1;
     return bpt / esz;
 }
@@ -504,7 +504,7 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
 
     long long nb = n_tiles + n_stiles;
     if (nb > max_blocks) nb = max_blocks;
-    const size_t smem = (size_t)kStages * rows_per_stage(S) * kThreads * cpt * esz;
+    const size_t smem = (size_t)kStages * rows_per_stage(ctx->dtype, S) * kThreads * cpt * esz;
     cudaError_t e = launch_reduce(fused, ctx->dtype, cpt, (int)nb, a, smem, s);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "launch of the reduce kernel");
     ctx->launches += 1;
@@ -625,7 +625,7 @@ adascale_status adascale_tiling(const int64_t *numel, int32_t n_tensors, int32_t
         sprefix[k] = sp[(size_t)k];
     }
     *tile_cols = kThreads * cpt;
-    *rows = rows_per_stage(S);
+    *rows = rows_per_stage(grad_dtype, S);
     return ADASCALE_OK;
 }
 

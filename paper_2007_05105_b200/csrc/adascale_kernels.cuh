@@ -35,7 +35,9 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kStagedThreads = kThreads + 32;  // + 1 producer warp
 constexpr int kStagedWarps = kStagedThreads / 32;
 constexpr int kStages = 3;                // shared-memory stages per block
-constexpr int kMaxRowsPerStage = 16;      // rows of one stage; larger S goes through in row chunks
+// Rows of one stage; larger S goes through in row chunks.  8 rows of 4 KB (fp32) and 16 rows of
+// 2 KB (bf16) were the fastest splits of a 32 KB stage in measurement.
+__host__ __device__ constexpr int max_rows_per_stage(int dtype) { return dtype == ADASCALE_BF16 ? 16 : 8; }
 constexpr int kStageBytes = 32 * 1024;    // upper bound of one stage
 constexpr int kReduceBlocksPerSM = 2;
 constexpr int kUpdateBlocksPerSM = 8;
@@ -540,7 +542,7 @@ __device__ __forceinline__ void store_cols(float *g, const float *m)
 // per row, completion counted on an mbarrier); eight consumer warps read them back.  Memory
 // latency is covered by the stages in flight rather than by registers, and the consumers
 // issue no global loads or address arithmetic.  A work item is (tile, row chunk):
-// kThreads * CPT columns of up to kMaxRowsPerStage rows.  Row chunks let any S through: the
+// kThreads * CPT columns of up to max_rows_per_stage rows.  Row chunks let any S through: the
 // per-column sums carry over from one chunk of rows to the next and close after the last.
 // ---------------------------------------------------------------------------------------
 //
@@ -564,7 +566,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const bool producer = warp == kStagedWarps - 1;
     const int S = a.S, T = a.T;
-    const int rps = S < kMaxRowsPerStage ? S : kMaxRowsPerStage;  // rows per stage
+    const int rps = S < max_rows_per_stage(DT) ? S : max_rows_per_stage(DT);  // rows per stage
     const int n_chunks = (S + rps - 1) / rps;
     const unsigned stage_bytes = (unsigned)rps * kRowBytes;
     const long long n_tiles = a.n_tiles;
