@@ -492,3 +492,30 @@ def test_steps_replayed_from_a_cuda_graph_match_eager_steps():
         assert torch.equal(a, b)
     eager.close()
     ada.close()
+
+
+def test_fused_mode_with_elastic_scale_host_gradients_and_resume():
+    gen = _gen(4300)
+    numels = [6000, 31]
+    lr = {"kind": "step", "eta0": 0.05, "d": 0.5, "milestones": (6.0,)}
+    pair = H.Pair(numels, 4, "bf16", momentum=0.9, weight_decay=1e-3, flags=FUSED, max_S=16, lr=lr)
+    w, v = _params(numels, gen)
+    pair.attach(w, v)
+    for S in (4, 8, 16, 2):
+        pair.dev.set_scale(S)
+        pair.orc.set_scale(S)
+        pair.step(_make_rows(numels, S, torch.bfloat16, gen), "fused elastic S=%d" % S)
+    # resume in a new context, and feed the next step from host memory
+    blob = pair.dev.get_state()
+    ada = B.AdaScale(numels, 2, "bf16", momentum=0.9, weight_decay=1e-3, flags=FUSED, max_S=16)
+    ada.set_state(blob)
+    rows = _make_rows(numels, 2, torch.bfloat16, gen)
+    w2, v2 = [t.clone() for t in w], [t.clone() for t in v]
+    pair.dev.step(rows, w, v, pair.sched_dev)
+    a = pair.dev.get_gain_tau(True).as_dict()
+    b = ada.step_host([[g.cpu().pin_memory() for g in row] for row in rows], w2, v2, pair.sched_dev).as_dict()
+    assert a == b
+    for x, y in zip(w + v, w2 + v2):
+        assert torch.equal(x, y)
+    ada.close()
+    pair.close()
