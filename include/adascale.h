@@ -172,6 +172,23 @@ adascale_status adascale_update(adascale_ctx *ctx, void *const *params, void *co
                                 void *cuda_stream);
 
 /*
+ * Column-sharded use on several GPUs (Sec. 2: the S workers' gradients are combined; here
+ * every GPU holds all S rows of ITS slice of the parameters, its own context over that
+ * slice, and the only exchange is the pair of sums).  adascale_reduce_sums is
+ * adascale_reduce without the scalar part: it writes the mean gradient of the slice and the
+ * slice's two sums, sums[0] = sum_i ||g_i - gbar||^2 and sums[1] = ||gbar||^2 (device
+ * pointer, 2 float64, 8-byte aligned), and leaves the state alone.  The caller adds the
+ * pairs of all GPUs (for instance an NCCL all-reduce of 16 bytes on the same stream), after
+ * which adascale_apply_sums runs the scalar part of App. B.3 / Eq. 3 / Sec. 3.2 on the
+ * completed sums and then the update of Eq. 2 for the slice.  Every GPU sees the identical
+ * two numbers and therefore computes the identical r_t, eta_t and tau.  Other arguments as in
+ * adascale_step.  Errors as there; ERR_STATE in the one-pass (fused) mode.
+ */
+adascale_status adascale_reduce_sums(adascale_ctx *ctx, const void *const *grads, void *sums, void *cuda_stream);
+adascale_status adascale_apply_sums(adascale_ctx *ctx, const void *sums, const adascale_lr_schedule *sched,
+                                    void *const *params, void *const *momentum, void *cuda_stream);
+
+/*
  * tau drives the caller's stopping test tau_t >= T_SI (Sec. 3.2); r_t and eta_t are what
  * the paper plots.  Copies the device state into *out (host pointer).  blocking != 0
  * waits for every step enqueued so far on the context's last stream; blocking == 0

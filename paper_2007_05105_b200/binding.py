@@ -20,7 +20,8 @@ STATUS_NONFINITE = 1
 MAX_MILESTONES = 8
 STATE_BYTES = 128
 
-EXPORTS = ("adascale_init", "adascale_step", "adascale_reduce", "adascale_update", "adascale_get_gain_tau",
+EXPORTS = ("adascale_init", "adascale_step", "adascale_reduce", "adascale_update", "adascale_reduce_sums",
+           "adascale_apply_sums", "adascale_get_gain_tau",
            "adascale_mean_grad", "adascale_set_scale", "adascale_get_state", "adascale_set_state",
            "adascale_step_host", "adascale_stream_probe", "adascale_tiling", "adascale_grad_stats_static", "adascale_launch_count",
            "adascale_destroy",
@@ -65,6 +66,8 @@ def _load():
     L.adascale_step.argtypes = [vp, vpp, vpp, vpp, C.POINTER(LrSchedule), vp]
     L.adascale_reduce.argtypes = [vp, vpp, C.POINTER(LrSchedule), vp]
     L.adascale_update.argtypes = [vp, vpp, vpp, vp]
+    L.adascale_reduce_sums.argtypes = [vp, vpp, vp, vp]
+    L.adascale_apply_sums.argtypes = [vp, vp, C.POINTER(LrSchedule), vpp, vpp, vp]
     L.adascale_get_gain_tau.argtypes = [vp, C.POINTER(Stats), C.c_int]
     L.adascale_mean_grad.argtypes = [vp, vpp]
     L.adascale_set_scale.argtypes = [vp, C.c_int32]
@@ -191,6 +194,16 @@ class AdaScale:
     def update(self, params, momentum, stream=None):
         self._check(lib.adascale_update(self._ctx, pointer_array(params), pointer_array(momentum),
                                         self._stream(stream)))
+
+    def reduce_sums(self, grads, sums, stream=None):
+        """Column-sharded use: this shard's mean gradient and its two sums (device float64[2])."""
+        self._check(lib.adascale_reduce_sums(self._ctx, pointer_array(grads), C.c_void_p(_ptr(sums)),
+                                             self._stream(stream)))
+
+    def apply_sums(self, sums, sched, params, momentum, stream=None):
+        """Scalar part on sums completed across shards, then this shard's update."""
+        self._check(lib.adascale_apply_sums(self._ctx, C.c_void_p(_ptr(sums)), C.byref(sched),
+                                            pointer_array(params), pointer_array(momentum), self._stream(stream)))
 
     def step_host(self, grads, params, momentum, sched, stream=None) -> Stats:
         out = Stats()

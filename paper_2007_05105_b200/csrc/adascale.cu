@@ -408,6 +408,20 @@ bool valid_sched(const adascale_lr_schedule *s)
     return true;
 }
 
+void fill_scalar_args(const adascale_ctx *ctx, const adascale_lr_schedule *sched, ScalarCfg &sc, Sched &out)
+{
+    sc.eps = ctx->eps;
+    sc.theta = resolve_theta(ctx);
+    sc.flags = ctx->flags;
+    sc.S = ctx->S;
+    out.kind = sched->kind;
+    out.n = sched->kind == ADASCALE_LR_STEP ? sched->n_milestones : 0;
+    out.eta0 = sched->eta0;
+    out.decay = sched->decay;
+    out.t_s1 = sched->t_s1;
+    for (int i = 0; i < ADASCALE_MAX_MILESTONES; ++i) out.w[i] = sched->milestones[i];
+}
+
 // Validates the caller's gradient pointers, rebuilds the tiling if the tile width or a tensor's
 // alignment changed, and uploads the pointer table ([max_S * T] row pointers).  Skipped entirely
 // when the pointers are those of the previous call.
@@ -462,7 +476,7 @@ adascale_status sync_reduce_table(adascale_ctx *ctx, const void *const *grads, c
 }
 
 adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const adascale_lr_schedule *sched,
-                          cudaStream_t s, bool fused)
+                          cudaStream_t s, bool fused, double *sums_out = nullptr)
 {
     const int S = ctx->S, T = ctx->T;
     const size_t esz = ctx->dtype == ADASCALE_BF16 ? 2 : 4;
@@ -487,20 +501,12 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
     a.partials = ctx->d_partials;
     a.ticket = ctx->d_ticket;
     a.st = ctx->d_state;
+    a.sums_out = sums_out;
     a.S = S;
     a.T = T;
     a.fS = (float)S;
     a.invS = 1.0f / (float)S;
-    a.sc.eps = ctx->eps;
-    a.sc.theta = resolve_theta(ctx);
-    a.sc.flags = ctx->flags;
-    a.sc.S = S;
-    a.sched.kind = sched->kind;
-    a.sched.n = sched->kind == ADASCALE_LR_STEP ? sched->n_milestones : 0;
-    a.sched.eta0 = sched->eta0;
-    a.sched.decay = sched->decay;
-    a.sched.t_s1 = sched->t_s1;
-    for (int i = 0; i < ADASCALE_MAX_MILESTONES; ++i) a.sched.w[i] = sched->milestones[i];
+    fill_scalar_args(ctx, sched, a.sc, a.sched);
 
     long long nb = n_tiles + n_stiles;
     if (nb > max_blocks) nb = max_blocks;
@@ -759,6 +765,48 @@ adascale_status adascale_update(adascale_ctx *ctx, void *const *params, void *co
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
     return do_update(ctx, params, momentum, (cudaStream_t)cuda_stream);
+}
+
+adascale_status adascale_reduce_sums(adascale_ctx *ctx, const void *const *grads, void *sums, void *cuda_stream)
+{
+    if (!ctx || !grads || !sums) return ADASCALE_ERR_INVALID_ARG;
+    if ((uintptr_t)sums % 8) return ADASCALE_ERR_ALIGNMENT;
+    if (ctx->flags & ADASCALE_FLAG_FUSED) return ADASCALE_ERR_STATE;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    if (ctx->P == 0) {  // no kernel runs for a shard without elements: its sums are zero
+        CU(cudaMemsetAsync(sums, 0, 2 * sizeof(double), s));
+        ctx->last_stream = s;
+        return ADASCALE_OK;
+    }
+    adascale_lr_schedule unused = {};
+    unused.kind = ADASCALE_LR_CONST;
+    unused.eta0 = 1.0;
+    return do_reduce(ctx, grads, &unused, s, false, static_cast<double *>(sums));
+}
+
+adascale_status adascale_apply_sums(adascale_ctx *ctx, const void *sums, const adascale_lr_schedule *sched,
+                                    void *const *params, void *const *momentum, void *cuda_stream)
+{
+    if (!ctx || !sums || !params || !momentum || !valid_sched(sched)) return ADASCALE_ERR_INVALID_ARG;
+    if ((uintptr_t)sums % 8) return ADASCALE_ERR_ALIGNMENT;
+    if (ctx->flags & ADASCALE_FLAG_FUSED) return ADASCALE_ERR_STATE;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    adascale_status st = sync_update_table(ctx, params, momentum, s);  // before anything is enqueued
+    if (st != ADASCALE_OK) return st;
+    ScalarArgs a;
+    a.st = ctx->d_state;
+    a.sums = static_cast<const double *>(sums);
+    fill_scalar_args(ctx, sched, a.sc, a.sched);
+    cudaError_t e = launch_overlapped(k_scalar, 1, 32, 0, s, a);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "launch of the scalar kernel");
+    ctx->launches += 1;
+    ctx->reduced = true;
+    ctx->last_stream = s;
+    return do_update(ctx, params, momentum, s);
 }
 
 adascale_status adascale_step(adascale_ctx *ctx, const void *const *grads, void *const *params,

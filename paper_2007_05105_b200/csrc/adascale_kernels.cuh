@@ -104,8 +104,17 @@ struct ReduceArgs {
     double2 *partials;
     unsigned *ticket;
     DevState *st;
+    double *sums_out;         // not null: write (D, N) there and leave the scalar part to k_scalar
     int S, T;
     float invS, fS;
+    ScalarCfg sc;
+    Sched sched;
+};
+
+// Scalar part on its own, for sums that were completed outside the reduce kernel.
+struct ScalarArgs {
+    DevState *st;
+    const double *sums;       // [0] = sum_i ||g_i - gbar||^2, [1] = ||gbar||^2, over ALL shards
     ScalarCfg sc;
     Sched sched;
 };
@@ -847,9 +856,24 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     }
     block_sum2<kStagedWarps>(d, n, sa, sb);
     if (tid == 0) {
-        scalar_step(a.st, a.sc, a.sched, d, n);
+        if (a.sums_out) {  // sharded use: the caller adds the shards' sums, k_scalar continues
+            a.sums_out[0] = d;
+            a.sums_out[1] = n;
+        } else {
+            scalar_step(a.st, a.sc, a.sched, d, n);
+        }
         *a.ticket = 0u;
     }
+}
+
+// Scalar part as a kernel of one thread: used when the two sums are completed outside the
+// reduce kernel (each GPU of a column-sharded job reduces its own columns, the sums are added
+// across GPUs, then every GPU runs the identical scalar step on the identical numbers).
+__global__ void k_scalar(const __grid_constant__ ScalarArgs a)
+{
+    griddep_launch();
+    griddep_wait();
+    if (threadIdx.x == 0 && blockIdx.x == 0) scalar_step(a.st, a.sc, a.sched, a.sums[0], a.sums[1]);
 }
 
 // ---------------------------------------------------------------------------------------

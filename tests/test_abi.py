@@ -79,6 +79,8 @@ def test_null_context_is_rejected_everywhere(B):
     assert B.lib.adascale_step(None, arr, arr, arr, C.byref(sched), None) == B.ERR_INVALID_ARG
     assert B.lib.adascale_reduce(None, arr, C.byref(sched), None) == B.ERR_INVALID_ARG
     assert B.lib.adascale_update(None, arr, arr, None) == B.ERR_INVALID_ARG
+    assert B.lib.adascale_reduce_sums(None, arr, arr, None) == B.ERR_INVALID_ARG
+    assert B.lib.adascale_apply_sums(None, arr, C.byref(sched), arr, arr, None) == B.ERR_INVALID_ARG
     assert B.lib.adascale_get_gain_tau(None, C.byref(st), 1) == B.ERR_INVALID_ARG
     assert B.lib.adascale_mean_grad(None, arr) == B.ERR_INVALID_ARG
     assert B.lib.adascale_set_scale(None, 2) == B.ERR_INVALID_ARG

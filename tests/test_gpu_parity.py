@@ -519,3 +519,43 @@ def test_fused_mode_with_elastic_scale_host_gradients_and_resume():
         assert torch.equal(x, y)
     ada.close()
     pair.close()
+
+
+def test_two_column_shards_reproduce_the_unsharded_step():
+    """Column-sharded use emulated on one GPU: two contexts over the two halves of the tensor
+    list, their sums added on the device (what an all-reduce of 16 bytes would do), then the
+    scalar part and the update per shard.  No kernel waits for another: the calls are sequential."""
+    gen = _gen(4400)
+    numels = [30000, 4097, 64, 7, 2048, 12345]
+    split = 3
+    steps = [_make_rows(numels, 8, torch.float32, gen, k=1.0 + i) for i in range(3)]
+    lr = {"kind": "exp", "eta0": 0.05, "d": 0.5, "T_S1": 10.0}
+    sched = H.device_lr(lr)
+
+    pair = H.Pair(numels, 8, "f32", momentum=0.9, weight_decay=1e-3, lr=lr)      # unsharded device + oracle
+    w, v = _params(numels, _gen(4401))
+    pair.attach(w, v)
+
+    ws, vs = _params(numels, _gen(4401))
+    shards = [B.AdaScale(numels[:split], 8, momentum=0.9, weight_decay=1e-3),
+              B.AdaScale(numels[split:], 8, momentum=0.9, weight_decay=1e-3)]
+    parts = [slice(0, split), slice(split, len(numels))]
+    sums = [torch.zeros(2, dtype=torch.float64, device=DEV) for _ in shards]
+    for i, rows in enumerate(steps):
+        pair._push_state = lambda tensors=None: None      # free-running here: compare the two device paths
+        st, ost = pair.step(rows, "unsharded step %d" % i, compare_tensors=False)
+        for ada, part, buf in zip(shards, parts, sums):
+            ada.reduce_sums([row[part] for row in rows], buf)
+        total = sums[0] + sums[1]                          # the exchange
+        for ada, part in zip(shards, parts):
+            ada.apply_sums(total, sched, ws[part], vs[part])
+        a, b = shards[0].get_gain_tau(True), shards[1].get_gain_tau(True)
+        assert a.as_dict() == b.as_dict()                  # every shard sees the identical scalars
+        for name in ("r", "tau", "eta", "sigma2_raw", "mu2_raw", "gbar_sqnorm", "dev_sqsum"):
+            assert getattr(a, name) == pytest.approx(getattr(st, name), rel=1e-12), name
+            assert getattr(a, name) == pytest.approx(ost[name] if name in ost else getattr(st, name), rel=1e-5)
+    for x, y in zip(w + v, ws + vs):
+        torch.testing.assert_close(x, y, rtol=1e-6, atol=1e-9)
+    for ada in shards:
+        ada.close()
+    pair.close()

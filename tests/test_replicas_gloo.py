@@ -55,3 +55,21 @@ def test_reference_arm_runs_on_rank_zero_only():
     line = json.loads(res.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["cpu_baseline"]["kind"] == "oracle"
     assert line["value"] > 0 and line["e2e"]["h2d_bytes_per_step"] == 0 and line["n_gpus"] == 2
+
+
+def _exchange_worker(rank, world, port, out_dir):
+    import torch
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    # the one exchange of the column-sharded path: each rank's (D, N) pair, summed over ranks
+    sums = torch.tensor([1.5 + rank, 0.25 * (rank + 1)], dtype=torch.float64)
+    dist.all_reduce(sums, op=dist.ReduceOp.SUM)
+    with open(os.path.join(out_dir, "s%d.json" % rank), "w") as f:
+        json.dump(sums.tolist(), f)
+    dist.destroy_process_group()
+
+
+def test_sharded_exchange_gives_every_rank_the_same_sums(tmp_path):
+    mp.spawn(_exchange_worker, args=(2, _free_port(), str(tmp_path)), nprocs=2, join=True)
+    got = [json.load(open(tmp_path / ("s%d.json" % r))) for r in range(2)]
+    assert got[0] == got[1] == [1.5 + 2.5, 0.25 + 0.5]
