@@ -26,8 +26,8 @@ if ROOT not in sys.path:
 METRIC = "adascale_step gradient GB/s and % of B200 HBM peak; step latency (us)"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the reduce kernel, from the ncu
 # captures summarised under profiles/ (same kernel build); None where no capture exists
-NCU_TRAFFIC_BYTES = {"resnet18": 383.4e6, "resnet50": 855.7e6}
-NCU_TRAFFIC_BYTES_FUSED = {"resnet18": 510.7e6}
+NCU_TRAFFIC_BYTES = {"resnet18": 382.5e6, "resnet50": 852.9e6}
+NCU_TRAFFIC_BYTES_FUSED = {"resnet18": 512.0e6}
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 L2_BYTES = 126 * 1024 * 1024
