@@ -248,6 +248,7 @@ def run_ours(args, wl):
                             T_S1=wl.lr.get("T_S1", 1.0), milestones=wl.lr.get("milestones", ()))
     gp, wp, vp = B.pointer_array(grads), B.pointer_array(w), B.pointer_array(v)
     stream = torch.cuda.current_stream(dev)
+    sh = stream.cuda_stream  # passed explicitly: no per-call stream lookup on the host
     working_set = wl.P * ((2 if wl.grad_dtype == "bf16" else 4) * wl.S + 12)
     flush = None
     if working_set <= 2 * L2_BYTES:
@@ -256,7 +257,7 @@ def run_ours(args, wl):
     def one_step():
         if flush is not None:
             flush.zero_()
-        ada.step(gp, wp, vp, sched)
+        ada.step(gp, wp, vp, sched, sh)
 
     for _ in range(warmup):
         one_step()
@@ -273,7 +274,7 @@ def run_ours(args, wl):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         for _ in range(steps):
-            ada.step(gp, wp, vp, sched)
+            ada.step(gp, wp, vp, sched, sh)
         e1.record(stream)
         torch.cuda.synchronize(dev)
         local_ms = e0.elapsed_time(e1) / steps
@@ -283,7 +284,7 @@ def run_ours(args, wl):
         for a, b in evs:
             flush.zero_()
             a.record(stream)
-            ada.step(gp, wp, vp, sched)
+            ada.step(gp, wp, vp, sched, sh)
             b.record(stream)
         torch.cuda.synchronize(dev)
         local_ms = sum(a.elapsed_time(b) for a, b in evs) / steps
@@ -301,12 +302,12 @@ def run_ours(args, wl):
             flush.zero_()
         a.record(stream)
         if fused:
-            ada.step(gp, wp, vp, sched)
+            ada.step(gp, wp, vp, sched, sh)
             b.record(stream)
         else:
-            ada.reduce(gp, sched)
+            ada.reduce(gp, sched, sh)
             b.record(stream)
-            ada.update(wp, vp)
+            ada.update(wp, vp, sh)
         c.record(stream)
     torch.cuda.synchronize(dev)
     t_reduce = sum(a.elapsed_time(b) for a, b, c in ev) / ksteps
@@ -314,7 +315,7 @@ def run_ours(args, wl):
     # the same kernels launched back to back on their own (no neighbour's dirty lines to write back)
     iso = {}
     if not fused:
-        for name, call in (("reduce", lambda: ada.reduce(gp, sched)), ("update", lambda: ada.update(wp, vp))):
+        for name, call in (("reduce", lambda: ada.reduce(gp, sched, sh)), ("update", lambda: ada.update(wp, vp, sh))):
             i0, i1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             for _ in range(3):
                 call()
@@ -330,7 +331,7 @@ def run_ours(args, wl):
         w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         w0.record(stream)
         for _ in range(steps):
-            ada.step(gp, wp, vp, sched)
+            ada.step(gp, wp, vp, sched, sh)
         w1.record(stream)
         torch.cuda.synchronize(dev)
         warm_ms = w0.elapsed_time(w1) / steps
