@@ -58,14 +58,14 @@ def test_every_element_is_covered_exactly_once(B, dtype):
 
 @pytest.mark.parametrize("name,S,dtype,expect_cols", [("resnet18", 8, "f32", 1024), ("resnet50", 16, "bf16", 1024),
                                                       ("transformer_base", 32, "f32", 1024),
-                                                      ("decoder_24l", 32, "bf16", 1024), ("single_1m", 4, "f32", 512)])
+                                                      ("decoder_24l", 32, "bf16", 1024), ("single_1m", 4, "f32", 1024)])
 def test_benchmark_workloads(B, name, S, dtype, expect_cols):
     from paper_2007_05105_b200 import synthetic
     numels = synthetic.workload(name).numels
     tp, sp, cols, rows = B.tiling(numels, S, dtype, None, 296)
     assert cols == expect_cols
     assert sp[-1] == 0                      # every benchmark tensor is a multiple of 8 elements
-    assert tp[-1] >= 4 * 296 or cols == 512  # enough tiles for every block, or the smallest tile
+    assert tp[-1] >= 2 * 296 or cols == 512  # two tiles for every block, or the smallest tile
     counts = [len(range(b, tp[-1], 296)) for b in range(296)]
     assert max(counts) - min(counts) <= 1
 
