@@ -34,6 +34,12 @@ MUTATIONS = [
     ("exponent not scaled by T_S1", "pow(lr->d, t / lr->T_S1)", "pow(lr->d, t)"),
     ("lagged r_0", ": 1.0;\n        st->n += 1;\n        st->avg_a = moving_average(st->avg_a, sigma2",
      ": 2.0;\n        st->n += 1;\n        st->avg_a = moving_average(st->avg_a, sigma2"),
+    ("ratio-mode r_0", "(st->avg_a + cfg->eps) / (st->avg_b + cfg->eps) : 1.0;",
+     "(st->avg_a + cfg->eps) / (st->avg_b + cfg->eps) : 2.0;"),
+    ("ratio-mode lagged gain taken after the update", "? r_prior\n                                              : (st->avg_a + cfg->eps)",
+     "? (st->avg_a + cfg->eps) / (st->avg_b + cfg->eps)\n                                              : (st->avg_a + cfg->eps)"),
+    ("ratio-mode eps missing from the lagged gain", "double r_prior = st->n > 0 ? (st->avg_a + cfg->eps) / (st->avg_b + cfg->eps)",
+     "double r_prior = st->n > 0 ? (st->avg_a) / (st->avg_b)"),
 ]
 
 

@@ -282,6 +282,58 @@ def test_lagged_mode_uses_prior_iterations_only(oracle_mod):
         prev = rc
 
 
+def test_lagged_ratio_estimator_uses_prior_iterations_only(oracle_mod):
+    """Sec. 3.4's estimator with App. B.3's lag: r_0 = 1, then the current-mode ratio gain of the iteration before."""
+    rng = np.random.default_rng(12)
+    S = 4
+    flags = oracle_mod.FLAG_RATIO
+    cur = oracle_mod.Oracle(S, theta=0.8, eps=0.25, flags=flags)
+    lag = oracle_mod.Oracle(S, theta=0.8, eps=0.25, flags=flags | oracle_mod.FLAG_LAGGED)
+    prev = 1.0  # r_0 = 1
+    taus = 0.0
+    for _ in range(12):
+        rows = _rows(rng, S, 30)
+        for o in (cur, lag):
+            o.reduce([[r] for r in rows])
+        rc = cur.scalar(oracle_mod.make_lr())["r"]
+        sl = lag.scalar(oracle_mod.make_lr())
+        assert sl["r"] == prev
+        taus += prev
+        assert sl["tau"] == pytest.approx(taus, rel=1e-15)
+        # both modes keep the same averages: only the gain that is read out lags
+        assert sl["avg_a"] == cur.state.avg_a and sl["avg_b"] == cur.state.avg_b
+        prev = rc
+
+
+def test_lagged_ratio_estimator_hand_worked(oracle_mod):
+    """Three iterations by hand, S = 2, theta = 1/2, eps = 1/2 (every value a dyadic rational).
+
+    m1 averages (1/S) sum_i ||g_i||^2, m2 averages ||gbar||^2, r = (m1 + eps) / (m2 + eps)   (Sec. 3.4),
+    read from the averages of prior iterations only, r_0 = 1   (App. B.3).
+    """
+    orc = oracle_mod.Oracle(2, theta=0.5, eps=0.5, flags=oracle_mod.FLAG_RATIO | oracle_mod.FLAG_LAGGED)
+    lr = oracle_mod.make_lr("const", eta0=2.0)
+    # iteration 0: samples (13, 8); no prior average -> r = 1; averages become (13, 8)
+    orc.reduce([[np.array([3.0, 4.0], np.float32)], [np.array([1.0, 0.0], np.float32)]])
+    st = orc.scalar(lr)
+    assert st["r"] == 1.0 and st["eta"] == 2.0 and st["tau"] == 1.0
+    assert (st["avg_a"], st["avg_b"]) == (13.0, 8.0)
+    # iteration 1: samples (2, 1); r from the prior averages = 13.5 / 8.5; the second sample is
+    # still inside the plain-mean warm-up: averages ((13 + 2)/2, (8 + 1)/2) = (7.5, 4.5)
+    orc.reduce([[np.array([1.0, 1.0], np.float32)], [np.array([1.0, -1.0], np.float32)]])
+    st = orc.scalar(lr)
+    assert st["r"] == pytest.approx(13.5 / 8.5, rel=1e-15)
+    assert st["eta"] == pytest.approx(27.0 / 8.5, rel=1e-15)
+    assert (st["avg_a"], st["avg_b"]) == (7.5, 4.5)
+    # iteration 2: r = (7.5 + 0.5) / (4.5 + 0.5) = 1.6 whatever this iteration's gradients are;
+    # samples (8, 8) enter with weight 1 - theta: averages (7.75, 6.25)
+    orc.reduce([[np.array([2.0, 2.0], np.float32)], [np.array([2.0, 2.0], np.float32)]])
+    st = orc.scalar(lr)
+    assert st["r"] == pytest.approx(1.6, rel=1e-15)
+    assert st["tau"] == pytest.approx(1.0 + 13.5 / 8.5 + 1.6, rel=1e-15)
+    assert (st["avg_a"], st["avg_b"]) == (7.75, 6.25)
+
+
 def test_elastic_scale_change_keeps_averages(oracle_mod):
     orc = oracle_mod.Oracle(2, theta=0.5)
     _feed(orc, oracle_mod, 4.0, 6.0)
