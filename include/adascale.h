@@ -82,6 +82,15 @@ typedef struct {
                                      (reduce, update, mean_grad return ERR_STATE), and non-finite
                                      gradients have already reached their own coordinates of w
                                      and v when they are detected (the state and tau still skip) */
+#define ADASCALE_FLAG_GRADS_READY 16u /* the caller vouches that every gradient row was completely
+                                     written before the step's first kernel can start: the rows were
+                                     produced on another stream and joined by an event, or the last
+                                     kernel before the step on `cuda_stream` does not trigger
+                                     programmatic dependent launches before its last gradient store
+                                     (kernels that never use that feature qualify).  The reduce kernel
+                                     then starts streaming the rows while the previous kernel in the
+                                     stream still drains.  Without the flag it waits for that kernel
+                                     first, which is always safe.  No counterpart in the paper.      */
 
 typedef struct {
     int32_t S;              /* scale: gradient rows per iteration, >= 1                */
@@ -100,8 +109,13 @@ typedef struct {
 
 /* status bits reported in adascale_stats.status_bits */
 #define ADASCALE_STATUS_NONFINITE 1u    /* last step saw inf/nan sums and was skipped           */
-#define ADASCALE_STATUS_WAIT_TIMEOUT 2u /* sticky: a bounded wait inside a kernel gave up; the
-                                           results of that step and later ones are not valid    */
+#define ADASCALE_STATUS_WAIT_TIMEOUT 2u /* sticky: a bounded wait inside the reduce kernel gave up.
+                                           That step and every later one is skipped: the state and
+                                           tau do not advance, `skipped` counts them, and w and v
+                                           stay as they were (one-pass mode: the tiles that the
+                                           kernel had reached before giving up are already updated).
+                                           The mean gradient of that step is incomplete.
+                                           adascale_set_state clears the condition.              */
 
 typedef struct {
     double r;           /* gain ratio r_t of the last step                            */
@@ -149,6 +163,9 @@ adascale_status adascale_init(const adascale_config *cfg, adascale_ctx **out);
  * that is refused with ERR_STATE (capture a step whose pointers were already seen).
  * A step whose sums are not finite changes nothing (state, tau, parameters, momentum)
  * and raises ADASCALE_STATUS_NONFINITE; this policy is an extension, the paper is silent.
+ * Ordering on the stream: the step's kernels are launched with programmatic dependent launch
+ * among themselves.  The gradient rows are read only after the kernel that precedes the step
+ * on `cuda_stream` has completed, unless cfg.flags carries ADASCALE_FLAG_GRADS_READY.
  */
 adascale_status adascale_step(adascale_ctx *ctx, const void *const *grads, void *const *params,
                               void *const *momentum, const adascale_lr_schedule *sched,
@@ -212,6 +229,17 @@ adascale_status adascale_mean_grad(adascale_ctx *ctx, const void **gbar);
 adascale_status adascale_set_scale(adascale_ctx *ctx, int32_t S);
 
 /*
+ * Every wait inside the reduce kernel (consumer warps waiting for a stage of rows, the producer
+ * warp waiting for a free stage) gives up after a number of polls and raises
+ * ADASCALE_STATUS_WAIT_TIMEOUT instead of hanging.  This sets that number for the following
+ * steps (default 4,194,304; 0 makes every such wait give up at once).  It exists so that the
+ * give-up path can be exercised by a test; the wait for copies that are already in flight when
+ * a block gives up keeps its own fixed bound, so a block never leaves while data is still
+ * arriving in its shared memory.  No counterpart in the paper.
+ */
+adascale_status adascale_set_wait_limit(adascale_ctx *ctx, uint32_t polls);
+
+/*
  * Checkpoint / resume of the scalar state (tau, averages, counters): buf is a host
  * buffer of ADASCALE_STATE_BYTES.  Both calls wait for the device.  set_state rejects a
  * buffer that get_state did not write (INVALID_ARG).  No counterpart in the paper.
@@ -263,10 +291,11 @@ adascale_status adascale_tiling(const int64_t *numel, int32_t n_tensors, int32_t
  * component that runs after start-up in a process where all device memory has already been
  * handed to another allocator, or one that must never risk the late failure or the implicit
  * device synchronisation that an allocation can bring.  Such a caller brings its own buffers
- * for inputs and outputs; what the kernel needs beyond them (a table of the row pointers,
- * a counter, one pair of partial sums per block, about 17 KB) sits in a fixed array inside
- * the library that every GPU which loads the library holds until the process exits.  The
- * call makes no cudaMalloc, cudaFree or other allocating call.
+ * for inputs and outputs; what the kernel needs beyond them (a counter and one pair of
+ * partial sums per block, about 16 KB) sits in a fixed array inside the library that every
+ * GPU which loads the library holds until the process exits.  The row pointers are passed to
+ * the kernel by value.  The call makes no cudaMalloc, cudaFree or other allocating call and
+ * copies nothing from host memory.
  *
  *   rows        host array [S] of device pointers, 16-byte aligned, n elements of grad_dtype each
  *   S           1 .. ADASCALE_STATIC_MAX_ROWS

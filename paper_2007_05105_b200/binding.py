@@ -15,14 +15,14 @@ LIB_PATH = os.path.join(_HERE, "libadascale_b200.so")
 OK, ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_CUDA, ERR_STATE, ERR_TOO_LARGE = range(6)
 F32, BF16 = 0, 1
 LR_CONST, LR_EXP, LR_STEP = 0, 1, 2
-FLAG_LAGGED, FLAG_CONT_TAU, FLAG_RATIO, FLAG_FUSED = 1, 2, 4, 8
-STATUS_NONFINITE = 1
+FLAG_LAGGED, FLAG_CONT_TAU, FLAG_RATIO, FLAG_FUSED, FLAG_GRADS_READY = 1, 2, 4, 8, 16
+STATUS_NONFINITE, STATUS_WAIT_TIMEOUT = 1, 2
 MAX_MILESTONES = 8
 STATE_BYTES = 128
 
 EXPORTS = ("adascale_init", "adascale_step", "adascale_reduce", "adascale_update", "adascale_reduce_sums",
            "adascale_apply_sums", "adascale_get_gain_tau",
-           "adascale_mean_grad", "adascale_set_scale", "adascale_get_state", "adascale_set_state",
+           "adascale_mean_grad", "adascale_set_scale", "adascale_set_wait_limit", "adascale_get_state", "adascale_set_state",
            "adascale_step_host", "adascale_stream_probe", "adascale_tiling", "adascale_grad_stats_static", "adascale_launch_count",
            "adascale_destroy",
            "adascale_strerror", "adascale_last_error")
@@ -71,6 +71,7 @@ def _load():
     L.adascale_get_gain_tau.argtypes = [vp, C.POINTER(Stats), C.c_int]
     L.adascale_mean_grad.argtypes = [vp, vpp]
     L.adascale_set_scale.argtypes = [vp, C.c_int32]
+    L.adascale_set_wait_limit.argtypes = [vp, C.c_uint32]
     L.adascale_get_state.argtypes = [vp, vp]
     L.adascale_set_state.argtypes = [vp, vp]
     L.adascale_step_host.argtypes = [vp, vpp, vpp, vpp, C.POINTER(LrSchedule), C.POINTER(Stats), vp]
@@ -237,6 +238,10 @@ class AdaScale:
     def set_scale(self, S):
         self._check(lib.adascale_set_scale(self._ctx, int(S)))
         self.S = int(S)
+
+    def set_wait_limit(self, polls):
+        """Bound of the reduce kernel's handshake waits (a test hook for the give-up path)."""
+        self._check(lib.adascale_set_wait_limit(self._ctx, int(polls)))
 
     def get_state(self) -> bytes:
         buf = C.create_string_buffer(STATE_BYTES)

@@ -8,21 +8,23 @@ namespace {
 // ---------------------------------------------------------------------------------------
 // Allocation-free variant of the reduce kernel for one tensor: the same shifted sums, the
 // same fp64 partials and fixed-order second stage, but rows are read with plain 128-bit loads
-// and everything the kernel needs besides its inputs and outputs (row-pointer table, ticket,
-// per-block partials) lives in one file-scope device array instead of memory from cudaMalloc.
+// and the scratch the kernel needs besides its inputs and outputs (ticket, per-block
+// partials) lives in one file-scope device array instead of memory from cudaMalloc.  The row
+// pointers travel by value in the kernel's parameters, so the call copies nothing from host
+// memory.
 // ---------------------------------------------------------------------------------------
 constexpr int kStaticMaxRows = ADASCALE_STATIC_MAX_ROWS;
 constexpr int kStaticMaxBlocks = 1024;
-constexpr size_t kStaticPtrBytes = 256;     // 32 row pointers
-constexpr size_t kStaticTicketOff = 256;    // one counter, padded to 256 bytes
-constexpr size_t kStaticPartialOff = 512;   // kStaticMaxBlocks pairs of doubles
+constexpr size_t kStaticTicketOff = 0;      // one counter, padded to 256 bytes
+constexpr size_t kStaticPartialOff = 256;   // kStaticMaxBlocks pairs of doubles
 constexpr size_t kStaticScratchBytes = kStaticPartialOff + kStaticMaxBlocks * sizeof(double2);
 
-// Shared by every call on this device and kept until the process exits (about 17 KB).
+// Shared by every call on this device and kept until the process exits (about 16 KB).
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 struct StaticArgs {
-    unsigned char *scratch;  // device address of g_static_scratch, resolved on the host
+    u64 rows[kStaticMaxRows];  // device addresses of the S rows
+    unsigned char *scratch;    // device address of g_static_scratch, resolved on the host
     float *gbar;
     double *sums;            // [0] = sum_i ||g_i - gbar||^2, [1] = ||gbar||^2
     long long n;
@@ -37,7 +39,7 @@ __global__ void __launch_bounds__(kThreads) k_grad_stats_static(const __grid_con
     __shared__ bool is_last;
     constexpr int E = Elem<DT>::kBytes;
     constexpr int V = 8;  // columns per thread and step
-    const u64 *rows = reinterpret_cast<const u64 *>(a.scratch);
+    const u64 *rows = a.rows;
     unsigned *ticket = reinterpret_cast<unsigned *>(a.scratch + kStaticTicketOff);
     double2 *partials = reinterpret_cast<double2 *>(a.scratch + kStaticPartialOff);
     const int tid = threadIdx.x, S = a.S;
@@ -179,6 +181,7 @@ struct adascale_ctx {
     DevState latest{};
     cudaStream_t last_stream = nullptr;
     bool reduced = false;
+    unsigned wait_spins = kSpinLimit;  // bound of the reduce kernel's handshake waits
     long long launches = 0;
     void *d_stage = nullptr;     // host-gradient staging (adascale_step_host)
     std::vector<const void *> stage_ptrs;
@@ -503,6 +506,8 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
     a.ticket = ctx->d_ticket;
     a.st = ctx->d_state;
     a.sums_out = sums_out;
+    a.spin_limit = ctx->wait_spins;
+    a.early_rows = (ctx->flags & ADASCALE_FLAG_GRADS_READY) ? 1u : 0u;
     a.S = S;
     a.T = T;
     a.fS = (float)S;
@@ -647,7 +652,8 @@ adascale_status adascale_init(const adascale_config *cfg, adascale_ctx **out)
     if (cfg->grad_dtype != ADASCALE_F32 && cfg->grad_dtype != ADASCALE_BF16) return ADASCALE_ERR_INVALID_ARG;
     if (!(cfg->theta < 1.0) || !(cfg->eps >= 0.0) || cfg->device < 0) return ADASCALE_ERR_INVALID_ARG;
     if (!std::isfinite(cfg->momentum) || !std::isfinite(cfg->weight_decay)) return ADASCALE_ERR_INVALID_ARG;
-    if (cfg->flags & ~(ADASCALE_FLAG_LAGGED | ADASCALE_FLAG_CONT_TAU | ADASCALE_FLAG_RATIO | ADASCALE_FLAG_FUSED))
+    if (cfg->flags & ~(ADASCALE_FLAG_LAGGED | ADASCALE_FLAG_CONT_TAU | ADASCALE_FLAG_RATIO | ADASCALE_FLAG_FUSED |
+                       ADASCALE_FLAG_GRADS_READY))
         return ADASCALE_ERR_INVALID_ARG;
     if ((cfg->flags & ADASCALE_FLAG_FUSED) && !(cfg->flags & ADASCALE_FLAG_LAGGED))
         return ADASCALE_ERR_INVALID_ARG;  // the one-pass form needs eta_t before the gradients are read
@@ -890,6 +896,13 @@ adascale_status adascale_set_scale(adascale_ctx *ctx, int32_t S)
     return ADASCALE_OK;
 }
 
+adascale_status adascale_set_wait_limit(adascale_ctx *ctx, uint32_t polls)
+{
+    if (!ctx) return ADASCALE_ERR_INVALID_ARG;
+    ctx->wait_spins = polls;
+    return ADASCALE_OK;
+}
+
 adascale_status adascale_get_state(adascale_ctx *ctx, void *buf)
 {
     if (!ctx || !buf) return ADASCALE_ERR_INVALID_ARG;
@@ -1058,14 +1071,11 @@ adascale_status adascale_grad_stats_static(const void *const *rows, int32_t S, i
         sms = sms_of[dev];
     }
 
-    // the row pointers go into the scratch array; the ticket must start at zero whatever the
-    // previous call left behind
-    u64 table[kStaticMaxRows] = {0};
-    for (int i = 0; i < S; ++i) table[i] = (u64)(uintptr_t)rows[i];
-    CU(cudaMemcpyAsync(scratch, table, kStaticPtrBytes, cudaMemcpyHostToDevice, s));  // pageable: staged before return
+    // the ticket must start at zero whatever the previous call left behind
     CU(cudaMemsetAsync(scratch + kStaticTicketOff, 0, sizeof(unsigned), s));
 
     StaticArgs a;
+    for (int i = 0; i < kStaticMaxRows; ++i) a.rows[i] = i < S ? (u64)(uintptr_t)rows[i] : 0;
     a.scratch = scratch;
     a.gbar = static_cast<float *>(gbar);
     a.sums = static_cast<double *>(sums);

@@ -46,7 +46,8 @@ constexpr int kUpdateTile = 1024;         // elements per tile of the update ker
 constexpr int kGbarAlign = 64;            // every tensor's mean gradient starts on a 256-byte boundary
 constexpr int kRing = 4;                  // pinned staging slots for pointer-table uploads
 constexpr int kMaxS = 4096;
-constexpr unsigned kSpinLimit = 1u << 22; // bounded waits: give up, flag, leave
+constexpr unsigned kSpinLimit = 1u << 22; // bounded waits: give up, flag, leave (default of the handshake waits,
+                                          // fixed bound of the wait for copies that are already in flight)
 
 typedef unsigned long long u64;
 
@@ -105,6 +106,8 @@ struct ReduceArgs {
     unsigned *ticket;
     DevState *st;
     double *sums_out;         // not null: write (D, N) there and leave the scalar part to k_scalar
+    unsigned spin_limit;      // bound of the producer / consumer handshake waits
+    unsigned early_rows;      // non-zero: the gradient rows may be read before griddepcontrol.wait
     int S, T;
     float invS, fS;
     ScalarCfg sc;
@@ -242,6 +245,11 @@ __device__ void scalar_step(DevState *st, const ScalarCfg &c, const Sched &sched
 {
     st->D = D;
     st->N = N;
+    if (__ldcg(&st->fault)) {  // a bounded wait gave up somewhere: the sums are incomplete, nothing is applied
+        st->skipped += 1;
+        st->eta = 0.0;
+        return;
+    }
     if (!isfinite(D) || !isfinite(N)) {  // skip the iteration, leave every average and tau alone
         st->status = ADASCALE_STATUS_NONFINITE;
         st->skipped += 1;
@@ -296,8 +304,6 @@ __device__ void scalar_step(DevState *st, const ScalarCfg &c, const Sched &sched
     st->t += 1;
 }
 
-// Persistent grid: every block walks its own segments and keeps two fp64 accumulators per
-// thread for the whole launch, so there is one block reduction and one partial pair per block.
 // Lagged estimate (App. B.3: r_t from the averages of prior iterations only, r_0 = 1): the
 // learning rate of the coming iteration is known before its gradients are read.  Same
 // expressions as in scalar_step, so both give the identical value.
@@ -316,6 +322,14 @@ __device__ double lagged_eta(const DevState *st, const ScalarCfg &c, const Sched
 // Programmatic dependent launch: a kernel lets its successor in the stream be scheduled
 // early, and waits for its predecessor (completion and visibility of its writes) only where
 // it first depends on it.  Both are no-ops for a launch without the attribute.
+//
+// Ordering rule of this library: a kernel triggers its dependents only AFTER its own
+// griddepcontrol.wait has returned.  A kernel can start no earlier than its predecessor's
+// trigger, so by induction, when a kernel of this library starts, every kernel that precedes
+// its predecessor in the stream has completed and its writes are visible.  What a kernel
+// touches before its own wait must therefore be data that its immediate predecessor does not
+// write: the update kernel's first w and v values (last written by the update before the
+// preceding reduce), and, only when the caller vouches for them, the gradient rows.
 __device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
@@ -333,11 +347,11 @@ __device__ __forceinline__ void mbar_expect_tx(u64 *bar, unsigned bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-// Returns false if the phase did not complete within the spin limit.
-__device__ __forceinline__ bool mbar_wait(u64 *bar, unsigned parity)
+// Returns false if the phase did not complete within `limit` polls.
+__device__ __forceinline__ bool mbar_wait(u64 *bar, unsigned parity, unsigned limit)
 {
     const unsigned addr = smem_u32(bar);
-    for (unsigned spin = 0; spin < kSpinLimit; ++spin) {
+    for (unsigned spin = 0; spin < limit; ++spin) {
         unsigned done;
         asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
                      : "=r"(done)
@@ -580,7 +594,6 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     const unsigned stage_bytes = (unsigned)rps * kRowBytes;
     const long long n_tiles = a.n_tiles;
 
-    griddep_launch();
     if (tid == 0) {
         for (int i = 0; i < kStages; ++i) {
             mbar_init(&full_bar[i], 1);
@@ -597,6 +610,13 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     bool timed_out = false;
 
     if (producer) {
+        // The rows are the caller's data.  Unless the caller has vouched that they were complete
+        // before this launch could start, the kernel before this one in the stream may be the one
+        // that writes them and may have triggered its dependents early: wait for it.
+        if (!a.early_rows) {
+            griddep_wait();
+            griddep_launch();
+        }
         u64 policy;
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
         int last_use[kStages];
@@ -624,7 +644,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
             for (int ch = 0; ch < n_chunks; ++ch, ++item) {
                 const int st = item % kStages;
                 const unsigned use = item / kStages;
-                if (!mbar_wait(&empty_bar[st], (use & 1u) ^ 1u)) { timed_out = true; break; }
+                if (!mbar_wait(&empty_bar[st], (use & 1u) ^ 1u, a.spin_limit)) { timed_out = true; break; }
                 const int r0 = ch * rps;
                 const int rows = S - r0 < rps ? S - r0 : rps;
                 if (lane == 0) mbar_expect_tx(&full_bar[st], (unsigned)rows * tc * E);
@@ -647,17 +667,24 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
             }
         }
         if (timed_out) atomicExch(&abort_flag, 1);
-        if (timed_out || *(volatile int *)&abort_flag) {
-            // leaving early: copies already issued must land before this block's shared memory is reused
+        // Every copy this warp has issued must have landed before the block may leave (its shared
+        // memory is handed to the next block): wait for the last use of each stage, with the long
+        // fixed bound whatever the handshake limit is.  In a normal run the consumers are waiting
+        // for the same phases, so this costs nothing.
 #pragma unroll
-            for (int i = 0; i < kStages; ++i)
-                if (last_use[i] >= 0) mbar_wait(&full_bar[i], (unsigned)last_use[i] & 1u);
+        for (int i = 0; i < kStages; ++i)
+            if (last_use[i] >= 0 && !mbar_wait(&full_bar[i], (unsigned)last_use[i] & 1u, kSpinLimit))
+                atomicExch(&abort_flag, 1);
+        if (a.early_rows) {  // every thread of the block has then passed its wait and triggered
+            griddep_wait();
+            griddep_launch();
         }
     } else {
-        // The producer above may already stream gradient rows while the previous kernel in the
-        // stream (the update that still reads the old mean gradient) drains; nothing may be
-        // written before it has finished.
+        // Nothing may be written before the previous kernel in the stream (the update that still
+        // reads the old mean gradient and the old eta) has finished.  Only then is the next
+        // kernel allowed to start (see the ordering rule above).
         griddep_wait();
+        griddep_launch();
         float eta = 0.f;
         if constexpr (FUSED) {
             if (tid == 0) eta_shared = (float)lagged_eta(a.st, a.sc, a.sched);
@@ -712,7 +739,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
             for (int ch = 0; ch < n_chunks; ++ch, ++item) {
                 const int st = item % kStages;
                 const unsigned use = item / kStages;
-                if (!mbar_wait(&full_bar[st], use & 1u)) { timed_out = true; break; }
+                if (!mbar_wait(&full_bar[st], use & 1u, a.spin_limit)) { timed_out = true; break; }
                 const int r0 = ch * rps;
                 const int rows = S - r0 < rps ? S - r0 : rps;
                 unsigned addr = lane_base + (unsigned)st * stage_bytes;
@@ -871,8 +898,8 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
 // across GPUs, then every GPU runs the identical scalar step on the identical numbers).
 __global__ void k_scalar(const __grid_constant__ ScalarArgs a)
 {
-    griddep_launch();
     griddep_wait();
+    griddep_launch();
     if (threadIdx.x == 0 && blockIdx.x == 0) scalar_step(a.st, a.sc, a.sched, a.sums[0], a.sums[1]);
 }
 
@@ -894,7 +921,6 @@ __device__ __forceinline__ void update4(float4 &ww, float4 &vv, const float4 &gg
 
 __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const __grid_constant__ UpdateArgs a)
 {
-    griddep_launch();
     const int tid = threadIdx.x, T = a.T;
     const long long n_tiles = a.n_tiles, G = gridDim.x;
     // descriptor two tiles ahead, the tensor's pointers one tile ahead (see the reduce kernel)
@@ -908,16 +934,21 @@ __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const _
         fl_n = a.wflags[d1.tensor];
     }
     if ((long long)blockIdx.x + G < n_tiles) d2 = a.tiles[blockIdx.x + G];
-    // w and v of the first tile do not depend on the reduce kernel: they are requested while it
-    // still drains; eta_t and the mean gradient are read only after the wait
+    // w and v of the first tile are requested while the reduce kernel still drains.  They were
+    // last written by the previous update, which had completed before any block of the reduce
+    // kernel triggered this launch (ordering rule above); the loads bypass L1 so that no line
+    // cached on this SM before that can be served.  eta_t and the mean gradient, which the
+    // reduce kernel writes, are read only after the wait.
     float4 w_first = make_float4(0.f, 0.f, 0.f, 0.f), v_first = w_first;
     const bool first_fast = (long long)blockIdx.x < n_tiles && (fl_n & 1u) && d1.len == kUpdateTile;
     if (first_fast) {
-        w_first = ((const float4 *)(wp_n + d1.first))[tid];
-        v_first = ((const float4 *)(vp_n + d1.first))[tid];
+        w_first = __ldcg((const float4 *)(wp_n + d1.first) + tid);
+        v_first = __ldcg((const float4 *)(vp_n + d1.first) + tid);
     }
     griddep_wait();
-    if (a.st->status & ADASCALE_STATUS_NONFINITE) return;
+    griddep_launch();
+    // a skipped iteration (non-finite sums, or a bounded wait that gave up) changes nothing
+    if ((a.st->status & ADASCALE_STATUS_NONFINITE) || a.st->fault) return;
     const float eta = (float)a.st->eta;
     for (long long t = blockIdx.x; t < n_tiles; t += G) {
         d0 = d1; wp = wp_n; vp = vp_n; fl = fl_n;

@@ -22,6 +22,35 @@ def _gen(seed):
     return g
 
 
+# Bounds evidence: every gradient, parameter and momentum tensor of these tests sits between two
+# guard zones of 256 poison bytes, and after each test the zones must be untouched.
+GUARD_BYTES = 256
+POISON = 0xA5
+_guards = []
+
+
+def _guarded(n, dtype, misalign=0):
+    """n elements of `dtype` starting `misalign` elements past a 256-byte boundary, poison on both sides."""
+    esz = torch.empty(0, dtype=dtype).element_size()
+    g = GUARD_BYTES // esz
+    whole = torch.empty(g + misalign + n + g, device=DEV, dtype=dtype)
+    raw = whole.view(torch.uint8)
+    raw[:(g + misalign) * esz] = POISON
+    raw[(g + misalign + n) * esz:] = POISON
+    _guards.append((raw, (g + misalign) * esz, (g + misalign + n) * esz))
+    return whole[g + misalign:g + misalign + n]
+
+
+@pytest.fixture(autouse=True)
+def _guard_zones_stay_intact():
+    _guards.clear()
+    yield
+    torch.cuda.synchronize()
+    for raw, lo, hi in _guards:
+        assert bool((raw[:lo] == POISON).all()) and bool((raw[hi:] == POISON).all()), "write outside a tensor"
+    _guards.clear()
+
+
 def _make_rows(numels, S, dtype, gen, k=3.0, mean_std=0.1, misalign=0):
     """Separate allocations per (row, tensor); `misalign` shifts every view by that many elements."""
     mean = [torch.empty(n, device=DEV).normal_(0, mean_std, generator=gen) for n in numels]
@@ -29,17 +58,19 @@ def _make_rows(numels, S, dtype, gen, k=3.0, mean_std=0.1, misalign=0):
     for _ in range(S):
         row = []
         for n, m in zip(numels, mean):
-            buf = torch.empty(n + misalign, device=DEV, dtype=torch.float32).normal_(0, 1, generator=gen)
-            full = torch.empty(n + misalign, device=DEV, dtype=dtype)
-            full[misalign:] = (m + k * mean_std * buf[misalign:]).to(dtype)
-            row.append(full[misalign:])
+            buf = torch.empty(n, device=DEV, dtype=torch.float32).normal_(0, 1, generator=gen)
+            t = _guarded(n, dtype, misalign)
+            t.copy_((m + k * mean_std * buf).to(dtype))
+            row.append(t)
         rows.append(row)
     return rows
 
 
 def _params(numels, gen, misalign=0):
-    w = [torch.empty(n + misalign, device=DEV).normal_(0, 1, generator=gen)[misalign:] for n in numels]
-    v = [torch.empty(n + misalign, device=DEV).normal_(0, 0.1, generator=gen)[misalign:] for n in numels]
+    w, v = [], []
+    for n in numels:
+        w.append(_guarded(n, torch.float32, misalign).normal_(0, 1, generator=gen))
+        v.append(_guarded(n, torch.float32, misalign).normal_(0, 0.1, generator=gen))
     return w, v
 
 
@@ -134,7 +165,8 @@ def test_heavy_tailed_noise():
 
 
 @pytest.mark.parametrize("flags", [0, B.FLAG_LAGGED, B.FLAG_RATIO, B.FLAG_RATIO | B.FLAG_LAGGED, B.FLAG_CONT_TAU])
-@pytest.mark.parametrize("theta", [-1.0, 0.0, 0.7])
+# the grid of App. C for S = 4: theta in {0, 1 - S/10, 1 - S/100, 1 - S/1000 (the rule, passed as -1), 1 - S/10000}
+@pytest.mark.parametrize("theta", [0.0, 0.6, 0.96, -1.0, 0.9996])
 def test_estimator_variants_and_theta(flags, theta):
     gen = _gen(11)
     numels = [5000, 129]

@@ -6,8 +6,10 @@ ruled out because it can fail late or stall the device).  ``adascale_grad_stats_
 serves them: inputs and outputs are the caller's buffers and the library's scratch is a fixed
 array inside the library.  This test calls it through the C ABI twice in a row, with different
 sizes, row counts and element types, and compares the mean gradient and the two sums with what
-``adascale_reduce`` produces for the same rows, within the tolerances of the parity tests.
-The file is named so that pytest collects it last.
+``adascale_reduce`` produces for the same rows, within the tolerances of the parity tests; a
+second test compares it with the CPU oracle over the corner sizes (one row, two rows, the
+largest row count, fewer elements than one vector) with poisoned guard zones around the
+caller's output buffers.  The file is named so that pytest collects it last.
 """
 import numpy as np
 import pytest
@@ -18,6 +20,8 @@ pytestmark = pytest.mark.gpu
 if not torch.cuda.is_available():
     pytest.skip("needs a CUDA device", allow_module_level=True)
 
+import oracle  # noqa: E402
+import _harness as H  # noqa: E402
 from paper_2007_05105_b200 import binding as B  # noqa: E402
 
 DEV = torch.device("cuda:0")
@@ -56,6 +60,43 @@ def test_static_entry_point_matches_the_context_api_twice_in_a_row():
         mean = torch.empty(n, device=DEV).normal_(0, 0.1, generator=gen)
         rows = [(mean + 0.3 * torch.empty(n, device=DEV).normal_(0, 1, generator=gen)).to(dtype) for _ in range(S)]
         _check(rows, n, name)
+
+
+GUARD = 256  # bytes of poison either side of an output buffer
+
+
+def _guarded(nbytes):
+    """A device byte buffer with 0xA5-filled guard zones; returns (whole, payload view)."""
+    whole = torch.full((nbytes + 2 * GUARD,), 0xA5, dtype=torch.uint8, device=DEV)
+    return whole, whole[GUARD:GUARD + nbytes]
+
+
+def _guards_intact(whole, nbytes):
+    return bool((whole[:GUARD] == 0xA5).all()) and bool((whole[GUARD + nbytes:] == 0xA5).all())
+
+
+@pytest.mark.parametrize("name", ["f32", "bf16"])
+@pytest.mark.parametrize("S", [1, 2, 3, 32])
+def test_static_entry_point_matches_the_oracle_at_the_corner_sizes(S, name):
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(500 + S)
+    dtype = torch.bfloat16 if name == "bf16" else torch.float32
+    for n in (1, 7, 8, 300007):
+        mean = torch.empty(n, device=DEV).normal_(0, 0.1, generator=gen)
+        rows = [(mean + 0.3 * torch.empty(n, device=DEV).normal_(0, 1, generator=gen)).to(dtype) for _ in range(S)]
+        gw, gpay = _guarded(4 * n)
+        sw, spay = _guarded(16)
+        B.grad_stats_static(rows, n, name, gpay.data_ptr(), spay.data_ptr())
+        torch.cuda.synchronize()
+        assert _guards_intact(gw, 4 * n) and _guards_intact(sw, 16), "write outside the caller's buffers"
+        gbar = gpay.view(torch.float32).cpu().numpy()
+        D, N = spay.view(torch.float64).tolist()
+        rows_np = [H.to_numpy_rows(r) for r in rows]
+        ogbar, oD, oN, oQ = oracle.grad_stats(rows_np, True, H.NTHREADS)
+        label = "S=%d n=%d %s" % (S, n, name)
+        assert abs(D - oD) <= 1e-5 * abs(oD) + 1e-12 * oQ, (label, D, oD)
+        assert abs(N - oN) <= 1e-5 * abs(oN) + 1e-12 * oQ, (label, N, oN)
+        H.check_gbar(gbar, ogbar, H.row_scale(rows_np), label, H.gbar_ulps(S))
 
 
 def test_static_entry_point_rejects_what_it_cannot_hold():
