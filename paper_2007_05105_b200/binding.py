@@ -56,11 +56,11 @@ class AdaScaleError(RuntimeError):
         self.status = status
 
 
-def _load():
-    if not os.path.exists(LIB_PATH):
+def _load(path=LIB_PATH):
+    if not os.path.exists(path):
         raise ImportError("%s is missing: build it with `python -m paper_2007_05105_b200.build` "
-                          "(there is no CPU fallback)" % LIB_PATH)
-    L = C.CDLL(LIB_PATH)
+                          "(there is no CPU fallback)" % path)
+    L = C.CDLL(path)
     vp, vpp = C.c_void_p, C.POINTER(C.c_void_p)
     L.adascale_init.argtypes = [C.POINTER(Config), C.POINTER(vp)]
     L.adascale_step.argtypes = [vp, vpp, vpp, vpp, C.POINTER(LrSchedule), vp]

@@ -170,7 +170,11 @@ struct adascale_ctx {
     std::vector<unsigned char> tiled_aligned;  // alignment flags and tile width the device descriptors were built for
     int tiled_cpt = 0;
     float *d_gbar = nullptr;
-    double2 *d_partials = nullptr;
+    double2 *d_partials = nullptr;        // per block (scalar-path tiles)
+    double2 *d_tile_partials = nullptr;   // per staged tile
+    double2 *d_group_partials = nullptr;  // per group of kGroupTiles staged tiles
+    unsigned *d_group_count = nullptr;
+    long long n_groups_cap = 0;
     unsigned *d_ticket = nullptr;
     DevState *d_state = nullptr;
     PtrTable tg, tw;
@@ -503,7 +507,11 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
     a.rho = (float)ctx->rho;
     a.lambda = (float)ctx->lambda;
     a.partials = ctx->d_partials;
+    a.tile_partials = ctx->d_tile_partials;
+    a.group_partials = ctx->d_group_partials;
+    a.group_count = ctx->d_group_count;
     a.ticket = ctx->d_ticket;
+    a.tile_counter = reinterpret_cast<u64 *>(ctx->d_ticket + 192);
     a.st = ctx->d_state;
     a.sums_out = sums_out;
     a.spin_limit = ctx->wait_spins;
@@ -567,6 +575,8 @@ adascale_status do_update(adascale_ctx *ctx, void *const *params, void *const *m
     a.n_tiles = n_tiles;
     a.gbar = ctx->d_gbar;
     a.st = ctx->d_state;
+    a.next_chunk = reinterpret_cast<u64 *>(ctx->d_ticket + 64);
+    a.exit_ticket = ctx->d_ticket + 128;
     a.T = T;
     a.rho = (float)ctx->rho;
     a.lambda = (float)ctx->lambda;
@@ -710,8 +720,13 @@ adascale_status adascale_init(const adascale_config *cfg, adascale_ctx **out)
         CU(cudaMalloc(&ctx->d_gbar, gbar_alloc * sizeof(float)));
         CU(cudaMemset(ctx->d_gbar, 0, gbar_alloc * sizeof(float)));
         CU(cudaMalloc(&ctx->d_partials, (size_t)(ctx->sms * kReduceBlocksPerSM + 1) * sizeof(double2)));
-        CU(cudaMalloc(&ctx->d_ticket, sizeof(unsigned)));
-        CU(cudaMemset(ctx->d_ticket, 0, sizeof(unsigned)));
+        ctx->n_groups_cap = rcap / kGroupTiles + 1;
+        CU(cudaMalloc(&ctx->d_tile_partials, (size_t)(rcap > 0 ? rcap : 1) * sizeof(double2)));
+        CU(cudaMalloc(&ctx->d_group_partials, (size_t)ctx->n_groups_cap * sizeof(double2)));
+        CU(cudaMalloc(&ctx->d_group_count, (size_t)ctx->n_groups_cap * sizeof(unsigned)));
+        CU(cudaMemset(ctx->d_group_count, 0, (size_t)ctx->n_groups_cap * sizeof(unsigned)));
+        CU(cudaMalloc(&ctx->d_ticket, 4 * 256));  // four counters, 256 bytes apart
+        CU(cudaMemset(ctx->d_ticket, 0, 4 * 256));
         CU(cudaMalloc(&ctx->d_state, sizeof(DevState)));
         CU(cudaMemset(ctx->d_state, 0, sizeof(DevState)));
         adascale_status s1 = table_alloc(ctx, ctx->tg, (size_t)ctx->max_S * T);
@@ -742,6 +757,9 @@ adascale_status adascale_destroy(adascale_ctx *ctx)
         cudaFree(ctx->d_utiles);
         cudaFree(ctx->d_gbar);
         cudaFree(ctx->d_partials);
+        cudaFree(ctx->d_tile_partials);
+        cudaFree(ctx->d_group_partials);
+        cudaFree(ctx->d_group_count);
         cudaFree(ctx->d_ticket);
         cudaFree(ctx->d_state);
         cudaFree(ctx->d_stage);
@@ -952,6 +970,9 @@ adascale_status adascale_set_state(adascale_ctx *ctx, const void *buf)
     d.lr = b.lr;
     CU(cudaStreamSynchronize(ctx->last_stream));
     CU(cudaMemcpy(ctx->d_state, &d, sizeof d, cudaMemcpyHostToDevice));
+    // a launch that gave up on a wait may have left its work counters half way
+    CU(cudaMemset(ctx->d_ticket, 0, 4 * 256));
+    CU(cudaMemset(ctx->d_group_count, 0, (size_t)ctx->n_groups_cap * sizeof(unsigned)));
     if (b.S != ctx->S) {
         ctx->S = b.S;
         ctx->tg.valid = false;

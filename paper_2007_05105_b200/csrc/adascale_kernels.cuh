@@ -35,19 +35,23 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kStagedThreads = kThreads + 32;  // + 1 producer warp
 constexpr int kStagedWarps = kStagedThreads / 32;
 constexpr int kStages = 3;                // shared-memory stages per block
-// Rows of one stage; larger S goes through in row chunks.  8 rows of 4 KB (fp32) and 16 rows of
-// 2 KB (bf16) were the fastest splits of a 32 KB stage in measurement.
-__host__ __device__ constexpr int max_rows_per_stage(int dtype) { return dtype == ADASCALE_BF16 ? 16 : 8; }
+// Rows of one stage; larger S goes through in row chunks.  Eight rows of up to 4 KB measured
+// fastest for both element types (bf16: 8 rows of 4 KB beat 16 rows of 2 KB once tiles were
+// handed out dynamically).
+__host__ __device__ constexpr int max_rows_per_stage(int) { return 8; }
 constexpr int kStageBytes = 32 * 1024;    // upper bound of one stage
 constexpr int kReduceBlocksPerSM = 2;
-constexpr int kUpdateBlocksPerSM = 8;
+constexpr int kUpdateVecs = 2;            // 128-bit accesses per array, thread and tile of the update kernel
+constexpr int kUpdateBlocksPerSM = 4;
+constexpr int kGroupTiles = 64;           // tiles whose sums are added up together (a multiple of 32)
 constexpr int kScalarTile = 2048;         // elements per tile on the unaligned / ragged-tail path
-constexpr int kUpdateTile = 1024;         // elements per tile of the update kernel: one 128-bit access per thread
+constexpr int kUpdateTile = 1024 * kUpdateVecs;  // elements per tile of the update kernel
 constexpr int kGbarAlign = 64;            // every tensor's mean gradient starts on a 256-byte boundary
 constexpr int kRing = 4;                  // pinned staging slots for pointer-table uploads
 constexpr int kMaxS = 4096;
 constexpr unsigned kSpinLimit = 1u << 22; // bounded waits: give up, flag, leave (default of the handshake waits,
                                           // fixed bound of the wait for copies that are already in flight)
+constexpr unsigned long long kWaitNs = 2000000000ull;  // and no wait lasts longer than two seconds
 
 typedef unsigned long long u64;
 
@@ -90,6 +94,16 @@ struct __align__(16) TileDesc {
     int pad[2];
 };
 
+// What the producer warp tells the consumers about the contents of a stage.
+struct StageInfo {
+    long long tile;   // index of the staged tile
+    long long first;  // first element within its tensor
+    long long goff;   // where its mean gradient lives
+    float *w, *v;     // fused mode: the tensor's parameters and momentum
+    unsigned wflag;   // fused mode: bit0: both 16-byte aligned
+    int len;          // columns; < 0: no tile follows
+};
+
 // Reduce kernel: a tensor whose S row pointers are 16-byte aligned contributes staged tiles of
 // kThreads * CPT columns for its first numel & ~7 elements and one scalar tile for the ragged
 // rest; any other tensor contributes only scalar tiles of kScalarTile elements.
@@ -102,8 +116,12 @@ struct ReduceArgs {
     const u64 *wv;            // fused mode only: [2 * T] parameters then momentum
     const unsigned *wflags;   // fused mode only: [T] bit0: both pointers 16-byte aligned
     float rho, lambda;        // fused mode only
-    double2 *partials;
+    double2 *partials;        // [grid] sums over each block's scalar-path tiles
+    double2 *tile_partials;   // [n_tiles] sums of each staged tile
+    double2 *group_partials;  // [ceil(n_tiles / kGroupTiles)] sums of each group of staged tiles
+    unsigned *group_count;    // [same] tiles of the group delivered so far; zero between launches
     unsigned *ticket;
+    u64 *tile_counter;        // staged tiles handed out beyond each block's first; zero between launches
     DevState *st;
     double *sums_out;         // not null: write (D, N) there and leave the scalar part to k_scalar
     unsigned spin_limit;      // bound of the producer / consumer handshake waits
@@ -129,6 +147,8 @@ struct UpdateArgs {
     long long n_tiles;
     const float *gbar;
     const DevState *st;
+    u64 *next_chunk;          // tiles handed out beyond each block's first; zero between launches
+    unsigned *exit_ticket;    // the block that leaves last resets both counters
     int T;
     float rho, lambda;
 };
@@ -347,10 +367,19 @@ __device__ __forceinline__ void mbar_expect_tx(u64 *bar, unsigned bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-// Returns false if the phase did not complete within `limit` polls.
+__device__ __forceinline__ u64 global_ns()
+{
+    u64 t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Returns false if the phase did not complete within `limit` polls or within kWaitNs of wall
+// time, whichever comes first (one poll can itself suspend the thread for a while, so a poll
+// count alone does not bound the time).
 __device__ __forceinline__ bool mbar_wait(u64 *bar, unsigned parity, unsigned limit)
 {
     const unsigned addr = smem_u32(bar);
+    u64 t0 = 0;
     for (unsigned spin = 0; spin < limit; ++spin) {
         unsigned done;
         asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
@@ -358,6 +387,11 @@ __device__ __forceinline__ bool mbar_wait(u64 *bar, unsigned parity, unsigned li
                      : "r"(addr), "r"(parity)
                      : "memory");
         if (done) return true;
+        if ((spin & 63u) == 63u) {
+            const u64 now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitNs) return false;
+        }
     }
     return false;
 }
@@ -578,6 +612,11 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
 {
     extern __shared__ __align__(128) unsigned char stage_mem[];
     __shared__ __align__(8) u64 full_bar[kStages], empty_bar[kStages];
+    __shared__ StageInfo stage_info[kStages];           // what the producer put into each stage
+    // A warp releases a stage before it delivers the tile's sums, so its fastest sibling can be
+    // delivering the tile kStages further on while it still owes its own: kStages + 1 slots.
+    __shared__ double2 tile_part[kStages + 1][kWarps];  // per-warp sums of the tiles in flight
+    __shared__ int tile_done[kStages + 1];              // consumer warps that have delivered theirs
     __shared__ double sa[kStagedWarps], sb[kStagedWarps];
     __shared__ bool is_last;
     __shared__ int abort_flag;
@@ -599,13 +638,14 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
             mbar_init(&full_bar[i], 1);
             mbar_init(&empty_bar[i], kWarps);
         }
+        for (int i = 0; i <= kStages; ++i) tile_done[i] = 0;
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
 
-    double accD = 0.0, accN = 0.0;
+    double accD = 0.0, accN = 0.0;  // scalar-path tiles only; staged tiles go through per-tile sums
     unsigned item = 0;  // running count of staged work items, identical in every thread
     bool timed_out = false;
 
@@ -622,32 +662,83 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
         int last_use[kStages];
 #pragma unroll
         for (int i = 0; i < kStages; ++i) last_use[i] = -1;
-        // Round-robin tiles make every block visit most tensors, so table misses must stay off
-        // the copy queue: the descriptor is fetched two tiles ahead and this lane's row pointer
-        // (row = lane when S <= 32) one tile ahead.
+        // Tile indices: the first is blockIdx.x, the rest come from the counter.  The counter is
+        // written by the previous reduce launch (which may still be running when this block starts,
+        // see the ordering rule), so it is touched only after the wait: a block that streams rows
+        // early requests its first tile, waits, and only then asks for further tiles.  The index is
+        // fetched two tiles ahead, the descriptor one tile ahead and this lane's row pointer
+        // (row = lane when S <= 32) one tile ahead, so no table miss delays a copy.
         const long long G = gridDim.x;
+        bool late_fetch = a.early_rows != 0;
+        bool waited = !late_fetch;  // griddepcontrol.wait has returned in this warp
+        long long t1 = n_tiles, t2 = n_tiles;
+        if (!late_fetch) {
+            long long f1 = 0, f2 = 0;
+            if (lane == 0) {
+                f1 = G + (long long)atomicAdd(a.tile_counter, 1ull);
+                f2 = G + (long long)atomicAdd(a.tile_counter, 1ull);
+            }
+            t1 = __shfl_sync(0xffffffffu, f1, 0);
+            t2 = __shfl_sync(0xffffffffu, f2, 0);
+        }
         TileDesc d0, d1 = {}, d2 = {};
         const char *rowptr = nullptr, *rowptr_n = nullptr;
-        if ((long long)blockIdx.x < n_tiles) d1 = a.tiles[blockIdx.x];
-        if ((long long)blockIdx.x + G < n_tiles) d2 = a.tiles[blockIdx.x + G];
-        if ((long long)blockIdx.x < n_tiles && lane < S) rowptr_n = (const char *)a.gptr[(size_t)lane * T + d1.tensor];
-        for (long long t = blockIdx.x; t < n_tiles && !timed_out; t += G) {
+        float *pw = nullptr, *pv = nullptr, *pw_n = nullptr, *pv_n = nullptr;  // fused mode, lane 0 only
+        unsigned pfl = 0, pfl_n = 0;
+        long long t = blockIdx.x;
+        if (t < n_tiles) d1 = a.tiles[t];
+        if (t1 < n_tiles) d2 = a.tiles[t1];
+        if (t < n_tiles && lane < S) rowptr_n = (const char *)a.gptr[(size_t)lane * T + d1.tensor];
+        if constexpr (FUSED) {
+            if (t < n_tiles && lane == 0) {
+                pw_n = (float *)a.wv[d1.tensor];
+                pv_n = (float *)a.wv[T + d1.tensor];
+                pfl_n = a.wflags[d1.tensor];
+            }
+        }
+        while (t < n_tiles && !timed_out) {
             d0 = d1;
             rowptr = rowptr_n;
+            pw = pw_n; pv = pv_n; pfl = pfl_n;
             d1 = d2;
-            if (t + 2 * G < n_tiles) d2 = a.tiles[t + 2 * G];
-            if (t + G < n_tiles && d1.tensor != d0.tensor && lane < S)
-                rowptr_n = (const char *)a.gptr[(size_t)lane * T + d1.tensor];
+            long long f3 = n_tiles;
+            if (lane == 0 && t2 < n_tiles) f3 = G + (long long)atomicAdd(a.tile_counter, 1ull);
+            if (t2 < n_tiles) d2 = a.tiles[t2];
+            if (t1 < n_tiles && d1.tensor != d0.tensor) {
+                if (lane < S) rowptr_n = (const char *)a.gptr[(size_t)lane * T + d1.tensor];
+                if constexpr (FUSED) {
+                    if (lane == 0) {
+                        pw_n = (float *)a.wv[d1.tensor];
+                        pv_n = (float *)a.wv[T + d1.tensor];
+                        pfl_n = a.wflags[d1.tensor];
+                    }
+                }
+            }
             const int k = d0.tensor;
             const long long c0 = d0.first;
             const int tc = d0.len;
             for (int ch = 0; ch < n_chunks; ++ch, ++item) {
                 const int st = item % kStages;
                 const unsigned use = item / kStages;
+                if (!waited && item >= (unsigned)kStages) {
+                    // reusing a stage needs the consumers, and they start only after the previous
+                    // kernel: from here on this warp's bounded waits must not count its run time
+                    griddep_wait();
+                    griddep_launch();
+                    waited = true;
+                }
                 if (!mbar_wait(&empty_bar[st], (use & 1u) ^ 1u, a.spin_limit)) { timed_out = true; break; }
                 const int r0 = ch * rps;
                 const int rows = S - r0 < rps ? S - r0 : rps;
-                if (lane == 0) mbar_expect_tx(&full_bar[st], (unsigned)rows * tc * E);
+                if (lane == 0) {
+                    StageInfo &si = stage_info[st];
+                    si.tile = t;
+                    si.first = d0.first;
+                    si.goff = d0.goff;
+                    si.len = tc;
+                    if constexpr (FUSED) { si.w = pw; si.v = pv; si.wflag = pfl; }
+                    mbar_expect_tx(&full_bar[st], (unsigned)rows * tc * E);  // releases the writes above
+                }
                 __syncwarp();
 #pragma unroll
                 for (int i = 0; i < kStages; ++i)
@@ -665,17 +756,64 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                     }
                 }
             }
+            if (late_fetch) {  // the first tile's rows are on their way: now the counter may be used
+                late_fetch = false;
+                if (!waited) {
+                    griddep_wait();
+                    griddep_launch();
+                    waited = true;
+                }
+                long long f1 = 0, f2 = 0;
+                if (lane == 0) {
+                    f1 = G + (long long)atomicAdd(a.tile_counter, 1ull);
+                    f2 = G + (long long)atomicAdd(a.tile_counter, 1ull);
+                    f3 = G + (long long)atomicAdd(a.tile_counter, 1ull);
+                }
+                t1 = __shfl_sync(0xffffffffu, f1, 0);
+                t2 = __shfl_sync(0xffffffffu, f2, 0);
+                if (t1 < n_tiles) {
+                    d1 = a.tiles[t1];
+                    if (lane < S) rowptr_n = (const char *)a.gptr[(size_t)lane * T + d1.tensor];
+                    if constexpr (FUSED) {
+                        if (lane == 0) {
+                            pw_n = (float *)a.wv[d1.tensor];
+                            pv_n = (float *)a.wv[T + d1.tensor];
+                            pfl_n = a.wflags[d1.tensor];
+                        }
+                    }
+                }
+                if (t2 < n_tiles) d2 = a.tiles[t2];
+            }
+            t = t1;
+            t1 = t2;
+            t2 = __shfl_sync(0xffffffffu, f3, 0);
+        }
+        if (!timed_out) {  // an end mark in the next stage tells the consumers that no tile follows
+            const int st = item % kStages;
+            const unsigned use = item / kStages;
+            if (mbar_wait(&empty_bar[st], (use & 1u) ^ 1u, a.spin_limit)) {
+                if (lane == 0) {
+                    stage_info[st].len = -1;
+                    mbar_arrive(&full_bar[st]);
+                }
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < kStages; ++i)
+                    if (i == st) last_use[i] = (int)use;  // the end mark is this stage's last phase
+            } else {
+                timed_out = true;
+            }
         }
         if (timed_out) atomicExch(&abort_flag, 1);
         // Every copy this warp has issued must have landed before the block may leave (its shared
-        // memory is handed to the next block): wait for the last use of each stage, with the long
+        // memory is handed to the next block): wait for the last phase of each stage, with the long
         // fixed bound whatever the handshake limit is.  In a normal run the consumers are waiting
         // for the same phases, so this costs nothing.
 #pragma unroll
         for (int i = 0; i < kStages; ++i)
             if (last_use[i] >= 0 && !mbar_wait(&full_bar[i], (unsigned)last_use[i] & 1u, kSpinLimit))
                 atomicExch(&abort_flag, 1);
-        if (a.early_rows) {  // every thread of the block has then passed its wait and triggered
+        if (!waited) {  // a block without a staged tile: every thread passes its wait and triggers
             griddep_wait();
             griddep_launch();
         }
@@ -694,38 +832,26 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
         constexpr int NP = CPT / 2;
         const u64 keep = l2_keep_policy();
         f2 c[NP], s1[NP], s2[NP], p1[NP];  // per-column state as packed pairs
-        const long long G = gridDim.x;
-        TileDesc d0, d1 = {};  // descriptor one tile ahead, as above
-        if ((long long)blockIdx.x < n_tiles) d1 = a.tiles[blockIdx.x];
-        // fused mode: the tile's parameter and momentum pointers, fetched one tile ahead as well
-        float *wp = nullptr, *vp = nullptr, *wp_n = nullptr, *vp_n = nullptr;
-        unsigned fl = 0, fl_n = 0;
-        if constexpr (FUSED) {
-            if ((long long)blockIdx.x < n_tiles) {
-                wp_n = (float *)a.wv[d1.tensor];
-                vp_n = (float *)a.wv[T + d1.tensor];
-                fl_n = a.wflags[d1.tensor];
-            }
-        }
         const unsigned lane_base = smem_u32(stage_mem) + (unsigned)tid * CPT * E;
-        for (long long t = blockIdx.x; t < n_tiles && !timed_out; t += G) {
-            d0 = d1;
-            if (t + G < n_tiles) d1 = a.tiles[t + G];
-            const int tc = d0.len;
+        unsigned tseq = 0;  // tiles this block has consumed
+        while (!timed_out) {
+            // the tile that the producer has put into the next stage, or its end mark
+            StageInfo si;
+            {
+                const int st = item % kStages;
+                if (!mbar_wait(&full_bar[st], (item / kStages) & 1u, a.spin_limit)) { timed_out = true; break; }
+                si = stage_info[st];
+            }
+            if (si.len < 0) break;
+            const int tc = si.len;
             const bool active = tid * CPT < tc;
             float wr[CPT], vr[CPT];  // fused mode: this thread's parameters and momentum, requested
             float *wt = nullptr, *vt = nullptr;  // before the rows are consumed so they arrive meanwhile
             bool vec_wv = false;
             if constexpr (FUSED) {
-                wp = wp_n; vp = vp_n; fl = fl_n;
-                if (t + G < n_tiles && d1.tensor != d0.tensor) {
-                    wp_n = (float *)a.wv[d1.tensor];
-                    vp_n = (float *)a.wv[T + d1.tensor];
-                    fl_n = a.wflags[d1.tensor];
-                }
-                wt = wp + d0.first + tid * CPT;
-                vt = vp + d0.first + tid * CPT;
-                vec_wv = (fl & 1u) != 0;
+                wt = si.w + si.first + tid * CPT;
+                vt = si.v + si.first + tid * CPT;
+                vec_wv = (si.wflag & 1u) != 0;
                 if (active) {
                     if (vec_wv) {
                         Cols<ADASCALE_F32, CPT>::load((const char *)wt, wr);
@@ -736,6 +862,8 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                     }
                 }
             }
+            bool tile_complete = false;
+            float dacc = 0.f, nacc = 0.f;
             for (int ch = 0; ch < n_chunks; ++ch, ++item) {
                 const int st = item % kStages;
                 const unsigned use = item / kStages;
@@ -795,9 +923,9 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&empty_bar[st]);  // this warp is done with the stage
+                if (ch == n_chunks - 1) tile_complete = true;
                 if (active && ch == n_chunks - 1) {
                     float m[CPT];
-                    float dacc = 0.f, nacc = 0.f;
 #pragma unroll
                     for (int j = 0; j < NP; ++j) {
                         float cc[2], ss1[2], ss2[2];
@@ -830,12 +958,63 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                             for (int j = 0; j < CPT; ++j) { vt[j] = vr[j]; wt[j] = wr[j]; }
                         }
                     } else {
-                        store_cols_keep<CPT>(a.gbar + d0.goff + tid * CPT, m, keep);
+                        store_cols_keep<CPT>(a.gbar + si.goff + tid * CPT, m, keep);
                     }
-                    accD += (double)dacc;
-                    accN += (double)nacc;
                 }
             }
+            if (!tile_complete) break;  // a wait gave up inside the tile
+            // The tile's two sums, in a fixed order whatever block and warp order they are formed in:
+            // lanes by a shuffle tree, warps 0..7 by the warp that delivers last, tiles by groups
+            // of kGroupTiles in index order (closed by whoever delivers the group's last tile),
+            // groups by the block that finishes last.
+            {
+                const double wd = warp_sum((double)dacc), wn = warp_sum((double)nacc);
+                const int slot = tseq % (kStages + 1);
+                int closes = 0;
+                if (lane == 0) {
+                    tile_part[slot][warp] = make_double2(wd, wn);
+                    __threadfence_block();
+                    if (atomicAdd(&tile_done[slot], 1) == kWarps - 1) {
+                        tile_done[slot] = 0;
+                        __threadfence_block();
+                        double D = 0.0, N = 0.0;
+#pragma unroll
+                        for (int w = 0; w < kWarps; ++w) {
+                            D += *(volatile double *)&tile_part[slot][w].x;
+                            N += *(volatile double *)&tile_part[slot][w].y;
+                        }
+                        a.tile_partials[si.tile] = make_double2(D, N);
+                        __threadfence();
+                        const long long g = si.tile / kGroupTiles;
+                        const long long left = n_tiles - g * kGroupTiles;
+                        const unsigned size = left < kGroupTiles ? (unsigned)left : (unsigned)kGroupTiles;
+                        if (atomicAdd(&a.group_count[g], 1u) == size - 1) closes = 1;
+                    }
+                }
+                closes = __shfl_sync(0xffffffffu, closes, 0);
+                if (closes) {  // this warp delivered the last tile of its group: add the group up
+                    __threadfence();
+                    const long long g = si.tile / kGroupTiles;
+                    const long long base = g * kGroupTiles;
+                    double D = 0.0, N = 0.0;
+#pragma unroll
+                    for (int h = 0; h < kGroupTiles / 32; ++h) {
+                        const long long i = base + h * 32 + lane;
+                        if (i < n_tiles) {
+                            const double2 p = __ldcg(&a.tile_partials[i]);
+                            D += p.x;
+                            N += p.y;
+                        }
+                    }
+                    D = warp_sum(D);
+                    N = warp_sum(N);
+                    if (lane == 0) {
+                        a.group_partials[g] = make_double2(D, N);
+                        a.group_count[g] = 0u;  // ready for the next launch
+                    }
+                }
+            }
+            ++tseq;
         }
         // ragged tails (< 8 elements) and tensors that are not 16-byte aligned: plain loads
         for (long long t = blockIdx.x; t < a.n_stiles; t += gridDim.x) {
@@ -861,6 +1040,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
         if (timed_out) atomicExch(&abort_flag, 1);
     }
 
+    // scalar-path tiles: one pair per block (their assignment to blocks is static)
     block_sum2<kStagedWarps>(accD, accN, sa, sb);
     if (tid == 0) {
         if (abort_flag) atomicOr(&a.st->fault, ADASCALE_STATUS_WAIT_TIMEOUT);
@@ -872,10 +1052,17 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     __syncthreads();
     if (!is_last) return;
 
-    // Second stage, fixed order: thread j adds partials j, j+288, ... in index order, then the
-    // same block tree.  The result depends on the tiling only, not on how blocks were scheduled.
+    // Last stage, fixed order: thread j adds the group sums j, j+288, ... in index order, then the
+    // per-block pairs of the scalar-path tiles likewise, then the block tree.  The result depends
+    // on the tiling only, not on which block processed which tile.
     __threadfence();
     double d = 0.0, n = 0.0;
+    const long long n_groups = (n_tiles + kGroupTiles - 1) / kGroupTiles;
+    for (long long i = tid; i < n_groups; i += kStagedThreads) {
+        const double2 p = __ldcg(&a.group_partials[i]);
+        d += p.x;
+        n += p.y;
+    }
     for (int i = tid; i < (int)gridDim.x; i += kStagedThreads) {
         const double2 p = __ldcg(&a.partials[i]);
         d += p.x;
@@ -890,8 +1077,10 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
             scalar_step(a.st, a.sc, a.sched, d, n);
         }
         *a.ticket = 0u;
+        *a.tile_counter = 0ull;
     }
 }
+
 
 // Scalar part as a kernel of one thread: used when the two sums are completed outside the
 // reduce kernel (each GPU of a column-sharded job reduces its own columns, the sums are added
@@ -904,8 +1093,7 @@ __global__ void k_scalar(const __grid_constant__ ScalarArgs a)
 }
 
 // ---------------------------------------------------------------------------------------
-// Update kernel (Eq. 2 with momentum): tiles of kUpdateTile elements, one 128-bit access per
-// array and thread, tiles dealt round-robin like in the reduce kernel.
+// Update kernel (Eq. 2 with momentum).
 // ---------------------------------------------------------------------------------------
 __device__ __forceinline__ void update4(float4 &ww, float4 &vv, const float4 &gg, float rho, float lambda, float eta)
 {
@@ -919,70 +1107,65 @@ __device__ __forceinline__ void update4(float4 &ww, float4 &vv, const float4 &gg
     ww.w = fmaf(-eta, vv.w, ww.w);
 }
 
+// A block's first tile is tile blockIdx.x; every further tile comes from a counter, so at any moment the blocks of the grid work on one
+// narrow, advancing window of the three arrays whatever the relative speed of the SMs (a
+// narrow window keeps DRAM pages and the read/write batches of the memory controller
+// efficient), and no SM idles at the end.  The counter value is fetched one tile ahead and the
+// descriptor of the next tile while the current one is processed.  A tile is kUpdateTile =
+// 1024 * C elements: C 128-bit accesses per array and thread, all requested before the first
+// is used.  The block that leaves last resets the counters for the next launch.
 __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const __grid_constant__ UpdateArgs a)
 {
+    constexpr int C = kUpdateVecs;
+    __shared__ long long s_next[2];
     const int tid = threadIdx.x, T = a.T;
     const long long n_tiles = a.n_tiles, G = gridDim.x;
-    // descriptor two tiles ahead, the tensor's pointers one tile ahead (see the reduce kernel)
-    TileDesc d0, d1 = {}, d2 = {};
-    float *wp = nullptr, *vp = nullptr, *wp_n = nullptr, *vp_n = nullptr;
-    unsigned fl = 0, fl_n = 0;
-    if ((long long)blockIdx.x < n_tiles) {
-        d1 = a.tiles[blockIdx.x];
-        wp_n = (float *)a.wv[d1.tensor];
-        vp_n = (float *)a.wv[T + d1.tensor];
-        fl_n = a.wflags[d1.tensor];
-    }
-    if ((long long)blockIdx.x + G < n_tiles) d2 = a.tiles[blockIdx.x + G];
-    // w and v of the first tile are requested while the reduce kernel still drains.  They were
-    // last written by the previous update, which had completed before any block of the reduce
-    // kernel triggered this launch (ordering rule above); the loads bypass L1 so that no line
-    // cached on this SM before that can be served.  eta_t and the mean gradient, which the
-    // reduce kernel writes, are read only after the wait.
-    float4 w_first = make_float4(0.f, 0.f, 0.f, 0.f), v_first = w_first;
-    const bool first_fast = (long long)blockIdx.x < n_tiles && (fl_n & 1u) && d1.len == kUpdateTile;
-    if (first_fast) {
-        w_first = __ldcg((const float4 *)(wp_n + d1.first) + tid);
-        v_first = __ldcg((const float4 *)(vp_n + d1.first) + tid);
-    }
+    long long c = blockIdx.x;
+    TileDesc d = {}, dn = {};
+    if (c < n_tiles) d = a.tiles[c];
     griddep_wait();
     griddep_launch();
-    // a skipped iteration (non-finite sums, or a bounded wait that gave up) changes nothing
-    if ((a.st->status & ADASCALE_STATUS_NONFINITE) || a.st->fault) return;
+    // the counter belongs to the update launches; it is touched only after the wait, so that even
+    // two update launches in a row cannot meet on it
+    if (tid == 0) s_next[0] = G + (long long)atomicAdd(a.next_chunk, 1ull);
+    const bool skip = (a.st->status & ADASCALE_STATUS_NONFINITE) || a.st->fault;
     const float eta = (float)a.st->eta;
-    for (long long t = blockIdx.x; t < n_tiles; t += G) {
-        d0 = d1; wp = wp_n; vp = vp_n; fl = fl_n;
-        d1 = d2;
-        if (t + 2 * G < n_tiles) d2 = a.tiles[t + 2 * G];
-        if (t + G < n_tiles && d1.tensor != d0.tensor) {
-            wp_n = (float *)a.wv[d1.tensor];
-            vp_n = (float *)a.wv[T + d1.tensor];
-            fl_n = a.wflags[d1.tensor];
-        }
-        const long long first = d0.first;
-        const int len = d0.len;
-        float *w = wp + first, *v = vp + first;
-        const float *g = a.gbar + d0.goff;
-        const bool vec = (fl & 1u) != 0;
-        if (vec && len == kUpdateTile) {
-            const bool have = first_fast && t == (long long)blockIdx.x;
-            const float4 gg = ((const float4 *)g)[tid];
-            float4 ww = have ? w_first : ((const float4 *)w)[tid];
-            float4 vv = have ? v_first : ((const float4 *)v)[tid];
-            update4(ww, vv, gg, a.rho, a.lambda, eta);
-            ((float4 *)v)[tid] = vv;
-            ((float4 *)w)[tid] = ww;
+    __syncthreads();
+    int buf = 0;
+    while (c < n_tiles && !skip) {
+        const long long nc = s_next[buf];
+        if (tid == 0 && nc < n_tiles) s_next[buf ^ 1] = G + (long long)atomicAdd(a.next_chunk, 1ull);
+        if (nc < n_tiles) dn = a.tiles[nc];
+        float *w = (float *)a.wv[d.tensor] + d.first;
+        float *v = (float *)a.wv[T + d.tensor] + d.first;
+        const float *g = a.gbar + d.goff;
+        const bool vec = (a.wflags[d.tensor] & 1u) != 0;
+        const int len = d.len;
+        if (vec && len == 1024 * C) {
+            float4 gg[C], ww[C], vv[C];
+#pragma unroll
+            for (int j = 0; j < C; ++j) {
+                gg[j] = ((const float4 *)g)[tid + j * kThreads];
+                ww[j] = ((const float4 *)w)[tid + j * kThreads];
+                vv[j] = ((const float4 *)v)[tid + j * kThreads];
+            }
+#pragma unroll
+            for (int j = 0; j < C; ++j) {
+                update4(ww[j], vv[j], gg[j], a.rho, a.lambda, eta);
+                ((float4 *)v)[tid + j * kThreads] = vv[j];
+                ((float4 *)w)[tid + j * kThreads] = ww[j];
+            }
         } else {
             int done = 0;
             if (vec) {
                 const int nv = len >> 2;
-                if (tid < nv) {
-                    const float4 gg = ((const float4 *)g)[tid];
-                    float4 ww = ((const float4 *)w)[tid];
-                    float4 vv = ((const float4 *)v)[tid];
-                    update4(ww, vv, gg, a.rho, a.lambda, eta);
-                    ((float4 *)v)[tid] = vv;
-                    ((float4 *)w)[tid] = ww;
+                for (int i = tid; i < nv; i += kThreads) {
+                    const float4 g4 = ((const float4 *)g)[i];
+                    float4 w4 = ((const float4 *)w)[i];
+                    float4 v4 = ((const float4 *)v)[i];
+                    update4(w4, v4, g4, a.rho, a.lambda, eta);
+                    ((float4 *)v)[i] = v4;
+                    ((float4 *)w)[i] = w4;
                 }
                 done = nv << 2;
             }
@@ -991,6 +1174,17 @@ __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const _
                 v[e] = vn;
                 w[e] = fmaf(-eta, vn, w[e]);
             }
+        }
+        __syncthreads();
+        c = nc;
+        buf ^= 1;
+        d = dn;
+    }
+    if (tid == 0) {
+        __threadfence();
+        if (atomicAdd(a.exit_ticket, 1u) == gridDim.x - 1) {
+            *a.next_chunk = 0ull;
+            *a.exit_ticket = 0u;
         }
     }
 }

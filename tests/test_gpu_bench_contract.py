@@ -20,7 +20,7 @@ def _run(*extra, workload="single_1m", env=None):
                           "--warmup", "3", "--no-sweep", *extra], capture_output=True, text=True, timeout=600, cwd=ROOT,
                          env=env)
     assert res.returncode == 0, res.stderr[-2000:]
-    lines = [l for l in res.stdout.splitlines() if l.strip()]
+    lines = [l for l in res.stdout.splitlines() if l.lstrip().startswith("{")]   # NCCL may log its version
     assert len(lines) == 1
     return json.loads(lines[0])
 
