@@ -43,7 +43,11 @@ constexpr int kStageBytes = 32 * 1024;    // upper bound of one stage
 constexpr int kReduceBlocksPerSM = 2;
 constexpr int kUpdateVecs = 2;            // 128-bit accesses per array, thread and tile of the update kernel
 constexpr int kUpdateBlocksPerSM = 4;
-constexpr int kGroupTiles = 64;           // tiles whose sums are added up together (a multiple of 32)
+constexpr long long kUpdateOverlapMaxTiles = 2048;  // update tiles (4M parameters) up to which the update kernel
+                                                    // is launched as a programmatic dependent of the reduce kernel
+constexpr long long kDynamicMinTiles = 32768;  // staged tiles from which they are handed out from a counter
+constexpr int kSlots = kStages + 1;       // tiles of a block whose sums can be on their way at once
+static_assert(kSlots == 4, "the producer keeps the tile index of each slot in four named registers");
 constexpr int kScalarTile = 2048;         // elements per tile on the unaligned / ragged-tail path
 constexpr int kUpdateTile = 1024 * kUpdateVecs;  // elements per tile of the update kernel
 constexpr int kGbarAlign = 64;            // every tensor's mean gradient starts on a 256-byte boundary
@@ -96,7 +100,6 @@ struct __align__(16) TileDesc {
 
 // What the producer warp tells the consumers about the contents of a stage.
 struct StageInfo {
-    long long tile;   // index of the staged tile
     long long first;  // first element within its tensor
     long long goff;   // where its mean gradient lives
     float *w, *v;     // fused mode: the tensor's parameters and momentum
@@ -117,11 +120,10 @@ struct ReduceArgs {
     const unsigned *wflags;   // fused mode only: [T] bit0: both pointers 16-byte aligned
     float rho, lambda;        // fused mode only
     double2 *partials;        // [grid] sums over each block's scalar-path tiles
-    double2 *tile_partials;   // [n_tiles] sums of each staged tile
-    double2 *group_partials;  // [ceil(n_tiles / kGroupTiles)] sums of each group of staged tiles
-    unsigned *group_count;    // [same] tiles of the group delivered so far; zero between launches
+    double2 *run_partials;    // sums of the staged tiles: one pair per run, or per block (run_tiles == 0)
+    long long run_tiles;      // consecutive staged tiles handed out together; 0: static assignment
     unsigned *ticket;
-    u64 *tile_counter;        // staged tiles handed out beyond each block's first; zero between launches
+    u64 *tile_counter;        // runs handed out beyond each block's first; zero between launches
     DevState *st;
     double *sums_out;         // not null: write (D, N) there and leave the scalar part to k_scalar
     unsigned spin_limit;      // bound of the producer / consumer handshake waits
@@ -613,10 +615,13 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     extern __shared__ __align__(128) unsigned char stage_mem[];
     __shared__ __align__(8) u64 full_bar[kStages], empty_bar[kStages];
     __shared__ StageInfo stage_info[kStages];           // what the producer put into each stage
-    // A warp releases a stage before it delivers the tile's sums, so its fastest sibling can be
-    // delivering the tile kStages further on while it still owes its own: kStages + 1 slots.
-    __shared__ double2 tile_part[kStages + 1][kWarps];  // per-warp sums of the tiles in flight
-    __shared__ int tile_done[kStages + 1];              // consumer warps that have delivered theirs
+    // Per-thread sums of the tiles in flight, handed from the consumer warps to the producer warp
+    // (which has the time to add them up in fp64; a shuffle tree in every consumer warp and tile,
+    // and any fence or atomic per tile, measured 5-40 % slower).  A warp releases a stage before it
+    // hands over the tile's sums, so its fastest sibling can be handing over the tile kStages
+    // further on while it still owes its own: kStages + 1 slots.
+    __shared__ float2 tile_part[kSlots][kThreads];
+    __shared__ __align__(8) u64 part_bar[kSlots];       // completes when all consumer warps have handed over
     __shared__ double sa[kStagedWarps], sb[kStagedWarps];
     __shared__ bool is_last;
     __shared__ int abort_flag;
@@ -638,14 +643,14 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
             mbar_init(&full_bar[i], 1);
             mbar_init(&empty_bar[i], kWarps);
         }
-        for (int i = 0; i <= kStages; ++i) tile_done[i] = 0;
+        for (int i = 0; i < kSlots; ++i) mbar_init(&part_bar[i], kWarps);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
 
-    double accD = 0.0, accN = 0.0;  // scalar-path tiles only; staged tiles go through per-tile sums
+    double accD = 0.0, accN = 0.0;  // scalar-path tiles only; staged tiles go through the producer warp
     unsigned item = 0;  // running count of staged work items, identical in every thread
     bool timed_out = false;
 
@@ -662,30 +667,51 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
         int last_use[kStages];
 #pragma unroll
         for (int i = 0; i < kStages; ++i) last_use[i] = -1;
-        // Tile indices: the first is blockIdx.x, the rest come from the counter.  The counter is
-        // written by the previous reduce launch (which may still be running when this block starts,
-        // see the ordering rule), so it is touched only after the wait: a block that streams rows
-        // early requests its first tile, waits, and only then asks for further tiles.  The index is
-        // fetched two tiles ahead, the descriptor one tile ahead and this lane's row pointer
-        // (row = lane when S <= 32) one tile ahead, so no table miss delays a copy.
+        // How tiles reach the blocks.  Small jobs (a.run_tiles == 0): statically, tile t belongs to
+        // block t mod grid.  Large jobs: in runs of a.run_tiles consecutive tiles; a block's first
+        // run is run blockIdx.x and every further one comes from a counter, so the blocks of the
+        // grid always work on one narrow, advancing window of the gradient matrix whatever the
+        // relative speed of the SMs (this keeps DRAM pages hot: 3-6 % on the largest jobs against
+        // the static assignment; nothing on small ones, where the extra pairs to add up at the end
+        // would cost more).  The counter is written by the previous reduce launch, which may still
+        // be running when this block starts (see the ordering rule), so it is touched only after
+        // the wait: a block that streams rows early requests its first tile, waits, and only then
+        // asks for further runs.  Run indices are fetched two runs ahead, the descriptor one tile
+        // ahead and this lane's row pointer (row = lane when S <= 32) one tile ahead, so no table
+        // miss delays a copy.
         const long long G = gridDim.x;
-        bool late_fetch = a.early_rows != 0;
-        bool waited = !late_fetch;  // griddepcontrol.wait has returned in this warp
-        long long t1 = n_tiles, t2 = n_tiles;
-        if (!late_fetch) {
-            long long f1 = 0, f2 = 0;
-            if (lane == 0) {
-                f1 = G + (long long)atomicAdd(a.tile_counter, 1ull);
-                f2 = G + (long long)atomicAdd(a.tile_counter, 1ull);
-            }
-            t1 = __shfl_sync(0xffffffffu, f1, 0);
-            t2 = __shfl_sync(0xffffffffu, f2, 0);
+        const long long R = a.run_tiles;       // 0: static assignment
+        const long long n_runs = R > 0 ? (n_tiles + R - 1) / R : 0;
+        bool late_fetch = a.early_rows != 0 && R > 0;
+        bool waited = a.early_rows == 0;  // griddepcontrol.wait has returned in this warp
+        long long rq0 = n_runs, rq1 = n_runs;  // the next two runs of this block
+        auto fetch_run = [&]() -> long long {   // lane 0 asks, everybody gets the answer
+            long long f = 0;
+            if (lane == 0) f = G + (long long)atomicAdd(a.tile_counter, 1ull);
+            return __shfl_sync(0xffffffffu, f, 0);
+        };
+        if (R > 0 && !late_fetch) {
+            rq0 = fetch_run();
+            rq1 = fetch_run();
         }
+        // the tile after `tile` in this block's sequence (n_tiles when there is none); consumes a
+        // prefetched run index at the end of a run
+        auto next_tile = [&](long long tile) -> long long {
+            if (tile >= n_tiles) return n_tiles;
+            if (R == 0) return tile + G < n_tiles ? tile + G : n_tiles;
+            if ((tile + 1) % R != 0 && tile + 1 < n_tiles) return tile + 1;
+            const long long r = rq0;
+            rq0 = rq1;
+            rq1 = (late_fetch || r >= n_runs) ? n_runs : fetch_run();
+            return r < n_runs ? r * R : n_tiles;
+        };
         TileDesc d0, d1 = {}, d2 = {};
         const char *rowptr = nullptr, *rowptr_n = nullptr;
         float *pw = nullptr, *pv = nullptr, *pw_n = nullptr, *pv_n = nullptr;  // fused mode, lane 0 only
         unsigned pfl = 0, pfl_n = 0;
-        long long t = blockIdx.x;
+        long long t = R > 0 ? ((long long)blockIdx.x < n_runs ? (long long)blockIdx.x * R : n_tiles)
+                            : ((long long)blockIdx.x < n_tiles ? (long long)blockIdx.x : n_tiles);
+        long long t1 = next_tile(t);
         if (t < n_tiles) d1 = a.tiles[t];
         if (t1 < n_tiles) d2 = a.tiles[t1];
         if (t < n_tiles && lane < S) rowptr_n = (const char *)a.gptr[(size_t)lane * T + d1.tensor];
@@ -696,13 +722,46 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                 pfl_n = a.wflags[d1.tensor];
             }
         }
+        // Sums of the staged tiles, in a fixed order whatever block and warp order they are formed
+        // in.  The consumers leave the 256 per-thread pairs of a tile in shared memory; lane l of
+        // this warp adds threads l, l+32, ... of every tile of a run (static assignment: of every
+        // tile of the block), in order, into its own fp64 pair; a shuffle tree adds the lanes at the
+        // end of the run and the result goes to run_partials[run] (static: [block]) with a plain
+        // store.  The block that finishes last adds those pairs in index order.  With runs, nothing
+        // depends on which block processed which run.
+        unsigned q = 0;                 // tiles this block has staged
+        long long qt0 = 0, qt1 = 0, qt2 = 0, qt3 = 0;  // their indices, by slot (kSlots = 4)
+        double runD = 0.0, runN = 0.0;  // this lane's share of the run being delivered
+        auto deliver = [&](unsigned seq) -> bool {
+            const int slot = seq % kSlots;
+            if (!mbar_wait(&part_bar[slot], (seq / kSlots) & 1u, a.spin_limit)) return false;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) {
+                const float2 e = tile_part[slot][w * 32 + lane];
+                runD += (double)e.x;
+                runN += (double)e.y;
+            }
+            if (R > 0) {
+                const long long tile = slot == 0 ? qt0 : (slot == 1 ? qt1 : (slot == 2 ? qt2 : qt3));
+                if ((tile + 1) % R == 0 || tile + 1 == n_tiles) {  // last tile of its run
+                    const double D = warp_sum(runD), N = warp_sum(runN);
+                    if (lane == 0) a.run_partials[tile / R] = make_double2(D, N);
+                    runD = runN = 0.0;
+                }
+            }
+            return true;
+        };
         while (t < n_tiles && !timed_out) {
+            {
+                const int slot = q % kSlots;
+                if (slot == 0) qt0 = t; else if (slot == 1) qt1 = t; else if (slot == 2) qt2 = t; else qt3 = t;
+            }
+            ++q;
             d0 = d1;
             rowptr = rowptr_n;
             pw = pw_n; pv = pv_n; pfl = pfl_n;
             d1 = d2;
-            long long f3 = n_tiles;
-            if (lane == 0 && t2 < n_tiles) f3 = G + (long long)atomicAdd(a.tile_counter, 1ull);
+            const long long t2 = next_tile(t1);
             if (t2 < n_tiles) d2 = a.tiles[t2];
             if (t1 < n_tiles && d1.tensor != d0.tensor) {
                 if (lane < S) rowptr_n = (const char *)a.gptr[(size_t)lane * T + d1.tensor];
@@ -732,7 +791,6 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                 const int rows = S - r0 < rps ? S - r0 : rps;
                 if (lane == 0) {
                     StageInfo &si = stage_info[st];
-                    si.tile = t;
                     si.first = d0.first;
                     si.goff = d0.goff;
                     si.len = tc;
@@ -756,6 +814,10 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                     }
                 }
             }
+            // With this tile staged, the sums of the tile kStages before it leave: its slot is the one
+            // the next tile's sums will use.
+            if (!timed_out && q >= (unsigned)kSlots && !deliver(q - kSlots)) timed_out = true;
+            long long t_next = t1, t1_next = t2;
             if (late_fetch) {  // the first tile's rows are on their way: now the counter may be used
                 late_fetch = false;
                 if (!waited) {
@@ -763,16 +825,13 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                     griddep_launch();
                     waited = true;
                 }
-                long long f1 = 0, f2 = 0;
-                if (lane == 0) {
-                    f1 = G + (long long)atomicAdd(a.tile_counter, 1ull);
-                    f2 = G + (long long)atomicAdd(a.tile_counter, 1ull);
-                    f3 = G + (long long)atomicAdd(a.tile_counter, 1ull);
-                }
-                t1 = __shfl_sync(0xffffffffu, f1, 0);
-                t2 = __shfl_sync(0xffffffffu, f2, 0);
-                if (t1 < n_tiles) {
-                    d1 = a.tiles[t1];
+                rq0 = fetch_run();
+                rq1 = fetch_run();
+                // the sequence was built without the counter: rebuild what follows this tile
+                t_next = next_tile(t);
+                t1_next = next_tile(t_next);
+                if (t_next < n_tiles) {
+                    d1 = a.tiles[t_next];
                     if (lane < S) rowptr_n = (const char *)a.gptr[(size_t)lane * T + d1.tensor];
                     if constexpr (FUSED) {
                         if (lane == 0) {
@@ -782,11 +841,10 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                         }
                     }
                 }
-                if (t2 < n_tiles) d2 = a.tiles[t2];
+                if (t1_next < n_tiles) d2 = a.tiles[t1_next];
             }
-            t = t1;
-            t1 = t2;
-            t2 = __shfl_sync(0xffffffffu, f3, 0);
+            t = t_next;
+            t1 = t1_next;
         }
         if (!timed_out) {  // an end mark in the next stage tells the consumers that no tile follows
             const int st = item % kStages;
@@ -803,6 +861,13 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
             } else {
                 timed_out = true;
             }
+        }
+        // the sums of the last tiles; with the static assignment, the block's one pair
+        for (unsigned seq = q >= (unsigned)kSlots ? q - kSlots + 1 : 0u; seq < q && !timed_out; ++seq)
+            if (!deliver(seq)) timed_out = true;
+        if (R == 0) {
+            const double D = warp_sum(runD), N = warp_sum(runN);
+            if (lane == 0) a.run_partials[blockIdx.x] = make_double2(D, N);
         }
         if (timed_out) atomicExch(&abort_flag, 1);
         // Every copy this warp has issued must have landed before the block may leave (its shared
@@ -963,56 +1028,12 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                 }
             }
             if (!tile_complete) break;  // a wait gave up inside the tile
-            // The tile's two sums, in a fixed order whatever block and warp order they are formed in:
-            // lanes by a shuffle tree, warps 0..7 by the warp that delivers last, tiles by groups
-            // of kGroupTiles in index order (closed by whoever delivers the group's last tile),
-            // groups by the block that finishes last.
+            // the thread's two sums over its columns of the tile go to the producer warp
             {
-                const double wd = warp_sum((double)dacc), wn = warp_sum((double)nacc);
-                const int slot = tseq % (kStages + 1);
-                int closes = 0;
-                if (lane == 0) {
-                    tile_part[slot][warp] = make_double2(wd, wn);
-                    __threadfence_block();
-                    if (atomicAdd(&tile_done[slot], 1) == kWarps - 1) {
-                        tile_done[slot] = 0;
-                        __threadfence_block();
-                        double D = 0.0, N = 0.0;
-#pragma unroll
-                        for (int w = 0; w < kWarps; ++w) {
-                            D += *(volatile double *)&tile_part[slot][w].x;
-                            N += *(volatile double *)&tile_part[slot][w].y;
-                        }
-                        a.tile_partials[si.tile] = make_double2(D, N);
-                        __threadfence();
-                        const long long g = si.tile / kGroupTiles;
-                        const long long left = n_tiles - g * kGroupTiles;
-                        const unsigned size = left < kGroupTiles ? (unsigned)left : (unsigned)kGroupTiles;
-                        if (atomicAdd(&a.group_count[g], 1u) == size - 1) closes = 1;
-                    }
-                }
-                closes = __shfl_sync(0xffffffffu, closes, 0);
-                if (closes) {  // this warp delivered the last tile of its group: add the group up
-                    __threadfence();
-                    const long long g = si.tile / kGroupTiles;
-                    const long long base = g * kGroupTiles;
-                    double D = 0.0, N = 0.0;
-#pragma unroll
-                    for (int h = 0; h < kGroupTiles / 32; ++h) {
-                        const long long i = base + h * 32 + lane;
-                        if (i < n_tiles) {
-                            const double2 p = __ldcg(&a.tile_partials[i]);
-                            D += p.x;
-                            N += p.y;
-                        }
-                    }
-                    D = warp_sum(D);
-                    N = warp_sum(N);
-                    if (lane == 0) {
-                        a.group_partials[g] = make_double2(D, N);
-                        a.group_count[g] = 0u;  // ready for the next launch
-                    }
-                }
+                const int slot = tseq % kSlots;
+                tile_part[slot][tid] = make_float2(dacc, nacc);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&part_bar[slot]);
             }
             ++tseq;
         }
@@ -1052,16 +1073,28 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     __syncthreads();
     if (!is_last) return;
 
-    // Last stage, fixed order: thread j adds the group sums j, j+288, ... in index order, then the
-    // per-block pairs of the scalar-path tiles likewise, then the block tree.  The result depends
-    // on the tiling only, not on which block processed which tile.
+    // Last stage, fixed order: thread j adds the pairs j, j+288, ... of the runs (or blocks) in
+    // index order, sixteen loads in flight at a time, then the per-block pairs of the scalar-path
+    // tiles likewise, then the block tree.  The result depends on the tiling only.
     __threadfence();
     double d = 0.0, n = 0.0;
-    const long long n_groups = (n_tiles + kGroupTiles - 1) / kGroupTiles;
-    for (long long i = tid; i < n_groups; i += kStagedThreads) {
-        const double2 p = __ldcg(&a.group_partials[i]);
-        d += p.x;
-        n += p.y;
+    const long long n_pairs = a.run_tiles > 0 ? (n_tiles + a.run_tiles - 1) / a.run_tiles
+                                              : (n_tiles < (long long)gridDim.x ? n_tiles : (long long)gridDim.x);
+    {
+        constexpr int U = 16;
+        long long i = tid;
+        for (; i + (U - 1) * (long long)kStagedThreads < n_pairs; i += U * (long long)kStagedThreads) {
+            double2 p[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) p[u] = __ldcg(&a.run_partials[i + u * (long long)kStagedThreads]);
+#pragma unroll
+            for (int u = 0; u < U; ++u) { d += p[u].x; n += p[u].y; }
+        }
+        for (; i < n_pairs; i += kStagedThreads) {
+            const double2 p = __ldcg(&a.run_partials[i]);
+            d += p.x;
+            n += p.y;
+        }
     }
     for (int i = tid; i < (int)gridDim.x; i += kStagedThreads) {
         const double2 p = __ldcg(&a.partials[i]);
