@@ -587,19 +587,7 @@ adascale_status do_update(adascale_ctx *ctx, void *const *params, void *const *m
     a.lambda = (float)ctx->lambda;
     long long nb = n_tiles;
     if (nb > (long long)ctx->sms * kUpdateBlocksPerSM) nb = (long long)ctx->sms * kUpdateBlocksPerSM;
-    // Large jobs: the update kernel is launched in plain stream order.  Launched as a programmatic
-    // dependent, its blocks land on SMs on which blocks of the reduce kernel still run; those SMs
-    // keep the reduce kernel's split of shared memory and L1 (nearly all shared memory) for as
-    // long as a block stays on them, which with tiles handed out from a counter is the whole
-    // update kernel: measured 6 % of the step on 355M parameters.  Small jobs gain more from
-    // the overlap of the launch than they lose.
-    cudaError_t e;
-    if (n_tiles <= kUpdateOverlapMaxTiles) {
-        e = launch_overlapped(k_update, (int)nb, kThreads, 0, s, a);
-    } else {
-        k_update<<<(unsigned)nb, kThreads, 0, s>>>(a);
-        e = cudaGetLastError();
-    }
+    cudaError_t e = launch_overlapped(k_update, (int)nb, kThreads, 0, s, a);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "launch of the update kernel");
     ctx->launches += 1;
     ctx->last_stream = s;

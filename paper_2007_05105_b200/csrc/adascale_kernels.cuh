@@ -43,8 +43,6 @@ constexpr int kStageBytes = 32 * 1024;    // upper bound of one stage
 constexpr int kReduceBlocksPerSM = 2;
 constexpr int kUpdateVecs = 2;            // 128-bit accesses per array, thread and tile of the update kernel
 constexpr int kUpdateBlocksPerSM = 4;
-constexpr long long kUpdateOverlapMaxTiles = 2048;  // update tiles (4M parameters) up to which the update kernel
-                                                    // is launched as a programmatic dependent of the reduce kernel
 constexpr long long kDynamicMinTiles = 32768;  // staged tiles from which they are handed out from a counter
 constexpr int kSlots = kStages + 1;       // tiles of a block whose sums can be on their way at once
 static_assert(kSlots == 4, "the producer keeps the tile index of each slot in four named registers");
@@ -637,6 +635,16 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     const int n_chunks = (S + rps - 1) / rps;
     const unsigned stage_bytes = (unsigned)rps * kRowBytes;
     const long long n_tiles = a.n_tiles;
+    // When the next kernel may start.  One-pass mode: the successor is another reduce launch, whose
+    // producer warps want to start early, so every thread triggers it as soon as its own wait has
+    // returned.  Two-kernel mode: the successor is the update kernel, and a block of it that lands
+    // on an SM where a reduce block still runs keeps that SM's split of shared memory and L1
+    // (hardly any L1) for its whole life, which costs the update kernel up to a quarter of its
+    // speed; so only the block that finishes last triggers it, when every other SM is already
+    // idle, and the launch still overlaps the last stage below.
+    auto trigger_early = [] {
+        if constexpr (FUSED) griddep_launch();
+    };
 
     if (tid == 0) {
         for (int i = 0; i < kStages; ++i) {
@@ -660,7 +668,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
         // that writes them and may have triggered its dependents early: wait for it.
         if (!a.early_rows) {
             griddep_wait();
-            griddep_launch();
+            trigger_early();
         }
         u64 policy;
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
@@ -783,7 +791,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                     // reusing a stage needs the consumers, and they start only after the previous
                     // kernel: from here on this warp's bounded waits must not count its run time
                     griddep_wait();
-                    griddep_launch();
+                    trigger_early();
                     waited = true;
                 }
                 if (!mbar_wait(&empty_bar[st], (use & 1u) ^ 1u, a.spin_limit)) { timed_out = true; break; }
@@ -822,7 +830,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                 late_fetch = false;
                 if (!waited) {
                     griddep_wait();
-                    griddep_launch();
+                    trigger_early();
                     waited = true;
                 }
                 rq0 = fetch_run();
@@ -880,14 +888,14 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                 atomicExch(&abort_flag, 1);
         if (!waited) {  // a block without a staged tile: every thread passes its wait and triggers
             griddep_wait();
-            griddep_launch();
+            trigger_early();
         }
     } else {
         // Nothing may be written before the previous kernel in the stream (the update that still
         // reads the old mean gradient and the old eta) has finished.  Only then is the next
         // kernel allowed to start (see the ordering rule above).
         griddep_wait();
-        griddep_launch();
+        trigger_early();
         float eta = 0.f;
         if constexpr (FUSED) {
             if (tid == 0) eta_shared = (float)lagged_eta(a.st, a.sc, a.sched);
@@ -1072,6 +1080,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     }
     __syncthreads();
     if (!is_last) return;
+    if constexpr (!FUSED) griddep_launch();
 
     // Last stage, fixed order: thread j adds the pairs j, j+288, ... of the runs (or blocks) in
     // index order, sixteen loads in flight at a time, then the per-block pairs of the scalar-path
