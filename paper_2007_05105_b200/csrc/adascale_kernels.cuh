@@ -34,7 +34,7 @@ constexpr int kThreads = 256;             // consumer threads of the reduce kern
 constexpr int kWarps = kThreads / 32;
 constexpr int kStagedThreads = kThreads + 32;  // + 1 producer warp
 constexpr int kStagedWarps = kStagedThreads / 32;
-constexpr int kStages = 3;                // shared-memory stages per block
+constexpr int kStages = 3;                // most shared-memory stages per block (a launch uses 2 or 3)
 // Rows of one stage; larger S goes through in row chunks.  Eight rows of up to 4 KB measured
 // fastest for both element types (bf16: 8 rows of 4 KB beat 16 rows of 2 KB once tiles were
 // handed out dynamically).
@@ -120,6 +120,7 @@ struct ReduceArgs {
     double2 *partials;        // [grid] sums over each block's scalar-path tiles
     double2 *run_partials;    // sums of the staged tiles: one pair per run, or per block (run_tiles == 0)
     long long run_tiles;      // consecutive staged tiles handed out together; 0: static assignment
+    unsigned stages;          // shared-memory stages in use, 2 .. kStages
     unsigned *ticket;
     u64 *tile_counter;        // runs handed out beyond each block's first; zero between launches
     DevState *st;
@@ -635,6 +636,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     const int n_chunks = (S + rps - 1) / rps;
     const unsigned stage_bytes = (unsigned)rps * kRowBytes;
     const long long n_tiles = a.n_tiles;
+    const unsigned nst = a.stages;  // stages in use: 2 with the static assignment, 3 with runs (measured)
     // When the next kernel may start.  One-pass mode: the successor is another reduce launch, whose
     // producer warps want to start early, so every thread triggers it as soon as its own wait has
     // returned.  Two-kernel mode: the successor is the update kernel, and a block of it that lands
@@ -785,9 +787,9 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
             const long long c0 = d0.first;
             const int tc = d0.len;
             for (int ch = 0; ch < n_chunks; ++ch, ++item) {
-                const int st = item % kStages;
-                const unsigned use = item / kStages;
-                if (!waited && item >= (unsigned)kStages) {
+                const int st = item % nst;
+                const unsigned use = item / nst;
+                if (!waited && item >= nst) {
                     // reusing a stage needs the consumers, and they start only after the previous
                     // kernel: from here on this warp's bounded waits must not count its run time
                     griddep_wait();
@@ -855,8 +857,8 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
             t1 = t1_next;
         }
         if (!timed_out) {  // an end mark in the next stage tells the consumers that no tile follows
-            const int st = item % kStages;
-            const unsigned use = item / kStages;
+            const int st = item % nst;
+            const unsigned use = item / nst;
             if (mbar_wait(&empty_bar[st], (use & 1u) ^ 1u, a.spin_limit)) {
                 if (lane == 0) {
                     stage_info[st].len = -1;
@@ -911,8 +913,8 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
             // the tile that the producer has put into the next stage, or its end mark
             StageInfo si;
             {
-                const int st = item % kStages;
-                if (!mbar_wait(&full_bar[st], (item / kStages) & 1u, a.spin_limit)) { timed_out = true; break; }
+                const int st = item % nst;
+                if (!mbar_wait(&full_bar[st], (item / nst) & 1u, a.spin_limit)) { timed_out = true; break; }
                 si = stage_info[st];
             }
             if (si.len < 0) break;
@@ -938,8 +940,8 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
             bool tile_complete = false;
             float dacc = 0.f, nacc = 0.f;
             for (int ch = 0; ch < n_chunks; ++ch, ++item) {
-                const int st = item % kStages;
-                const unsigned use = item / kStages;
+                const int st = item % nst;
+                const unsigned use = item / nst;
                 if (!mbar_wait(&full_bar[st], use & 1u, a.spin_limit)) { timed_out = true; break; }
                 const int r0 = ch * rps;
                 const int rows = S - r0 < rps ? S - r0 : rps;
