@@ -142,6 +142,11 @@ def workload(name: str, **over) -> Workload:
     elif name == "decoder_24l":
         w = Workload(name, decoder_24l_shapes(), S=32, grad_dtype="bf16", k=(0.1, 10.0), steps=200,
                      lr={"kind": "exp", "eta0": 0.1, "d": 0.05, "T_S1": 5000.0}, seed=2007051055)
+    elif name == "decoder_4l":
+        # decoder_24l cut to 4 layers and a 16k vocabulary (68M parameters, 4.4 GB of gradients): small
+        # enough for a profiler capture, large enough to take the same kernel paths as decoder_24l
+        w = Workload(name, decoder_24l_shapes(layers=4, vocab=16384), S=32, grad_dtype="bf16", k=(0.1, 10.0), steps=200,
+                     lr={"kind": "exp", "eta0": 0.1, "d": 0.05, "T_S1": 5000.0}, seed=2007051056)
     else:
         raise KeyError(name)
     for key, val in over.items():
