@@ -118,7 +118,7 @@ struct ReduceArgs {
     const unsigned *wflags;   // fused mode only: [T] bit0: both pointers 16-byte aligned
     float rho, lambda;        // fused mode only
     double2 *partials;        // [grid] sums over each block's scalar-path tiles
-    double2 *run_partials;    // sums of the staged tiles: one pair per run, or per block (run_tiles == 0)
+    double2 *run_partials;    // sums of the staged tiles, one pair per run (run_tiles > 0)
     long long run_tiles;      // consecutive staged tiles handed out together; 0: static assignment
     unsigned stages;          // shared-memory stages in use, 2 .. kStages
     unsigned *ticket;
@@ -660,7 +660,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     }
     __syncthreads();
 
-    double accD = 0.0, accN = 0.0;  // scalar-path tiles only; staged tiles go through the producer warp
+    double accD = 0.0, accN = 0.0;  // scalar-path tiles, and the staged tiles of the static assignment
     unsigned item = 0;  // running count of staged work items, identical in every thread
     bool timed_out = false;
 
@@ -734,11 +734,11 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
         }
         // Sums of the staged tiles, in a fixed order whatever block and warp order they are formed
         // in.  The consumers leave the 256 per-thread pairs of a tile in shared memory; lane l of
-        // this warp adds threads l, l+32, ... of every tile of a run (static assignment: of every
-        // tile of the block), in order, into its own fp64 pair; a shuffle tree adds the lanes at the
-        // end of the run and the result goes to run_partials[run] (static: [block]) with a plain
-        // store.  The block that finishes last adds those pairs in index order.  With runs, nothing
-        // depends on which block processed which run.
+        // this warp adds threads l, l+32, ... of every tile of a run, in order, into its own fp64
+        // pair; a shuffle tree adds the lanes at the end of the run and the result goes to
+        // run_partials[run] with a plain store.  The block that finishes last adds those pairs in
+        // index order, so nothing depends on which block processed which run.  (Static assignment:
+        // none of this; the consumer threads keep their own fp64 pairs, see below.)
         unsigned q = 0;                 // tiles this block has staged
         long long qt0 = 0, qt1 = 0, qt2 = 0, qt3 = 0;  // their indices, by slot (kSlots = 4)
         double runD = 0.0, runN = 0.0;  // this lane's share of the run being delivered
@@ -826,7 +826,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
             }
             // With this tile staged, the sums of the tile kStages before it leave: its slot is the one
             // the next tile's sums will use.
-            if (!timed_out && q >= (unsigned)kSlots && !deliver(q - kSlots)) timed_out = true;
+            if (R > 0 && !timed_out && q >= (unsigned)kSlots && !deliver(q - kSlots)) timed_out = true;
             long long t_next = t1, t1_next = t2;
             if (late_fetch) {  // the first tile's rows are on their way: now the counter may be used
                 late_fetch = false;
@@ -873,12 +873,8 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
             }
         }
         // the sums of the last tiles; with the static assignment, the block's one pair
-        for (unsigned seq = q >= (unsigned)kSlots ? q - kSlots + 1 : 0u; seq < q && !timed_out; ++seq)
+        for (unsigned seq = q >= (unsigned)kSlots ? q - kSlots + 1 : 0u; R > 0 && seq < q && !timed_out; ++seq)
             if (!deliver(seq)) timed_out = true;
-        if (R == 0) {
-            const double D = warp_sum(runD), N = warp_sum(runN);
-            if (lane == 0) a.run_partials[blockIdx.x] = make_double2(D, N);
-        }
         if (timed_out) atomicExch(&abort_flag, 1);
         // Every copy this warp has issued must have landed before the block may leave (its shared
         // memory is handed to the next block): wait for the last phase of each stage, with the long
@@ -1038,12 +1034,18 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                 }
             }
             if (!tile_complete) break;  // a wait gave up inside the tile
-            // the thread's two sums over its columns of the tile go to the producer warp
-            {
+            if (a.run_tiles > 0) {
+                // runs from the counter: the thread's two sums over its columns of the tile go to
+                // the producer warp, which adds them up per run
                 const int slot = tseq % kSlots;
                 tile_part[slot][tid] = make_float2(dacc, nacc);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&part_bar[slot]);
+            } else {
+                // static assignment: the block's tiles are fixed, so the thread keeps its own fp64 pair
+                // for the whole launch and the block adds its threads up once, below
+                accD += (double)dacc;
+                accN += (double)nacc;
             }
             ++tseq;
         }
@@ -1071,7 +1073,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
         if (timed_out) atomicExch(&abort_flag, 1);
     }
 
-    // scalar-path tiles: one pair per block (their assignment to blocks is static)
+    // statically assigned tiles (all scalar-path tiles, the staged ones of small jobs): one pair per block
     block_sum2<kStagedWarps>(accD, accN, sa, sb);
     if (tid == 0) {
         if (abort_flag) atomicOr(&a.st->fault, ADASCALE_STATUS_WAIT_TIMEOUT);
@@ -1084,13 +1086,11 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     if (!is_last) return;
     if constexpr (!FUSED) griddep_launch();
 
-    // Last stage, fixed order: thread j adds the pairs j, j+288, ... of the runs (or blocks) in
-    // index order, sixteen loads in flight at a time, then the per-block pairs of the scalar-path
-    // tiles likewise, then the block tree.  The result depends on the tiling only.
+    // Last stage, fixed order: thread j adds the pairs j, j+288, ... of the runs in index order,
+    // sixteen loads in flight at a time, then the per-block pairs likewise, then the block tree.
     __threadfence();
     double d = 0.0, n = 0.0;
-    const long long n_pairs = a.run_tiles > 0 ? (n_tiles + a.run_tiles - 1) / a.run_tiles
-                                              : (n_tiles < (long long)gridDim.x ? n_tiles : (long long)gridDim.x);
+    const long long n_pairs = a.run_tiles > 0 ? (n_tiles + a.run_tiles - 1) / a.run_tiles : 0;
     {
         constexpr int U = 16;
         long long i = tid;
