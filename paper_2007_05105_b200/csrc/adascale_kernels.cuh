@@ -665,13 +665,6 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     bool timed_out = false;
 
     if (producer) {
-        // The rows are the caller's data.  Unless the caller has vouched that they were complete
-        // before this launch could start, the kernel before this one in the stream may be the one
-        // that writes them and may have triggered its dependents early: wait for it.
-        if (!a.early_rows) {
-            griddep_wait();
-            trigger_early();
-        }
         u64 policy;
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
         int last_use[kStages];
@@ -692,18 +685,20 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
         const long long G = gridDim.x;
         const long long R = a.run_tiles;       // 0: static assignment
         const long long n_runs = R > 0 ? (n_tiles + R - 1) / R : 0;
-        bool late_fetch = a.early_rows != 0 && R > 0;
-        bool waited = a.early_rows == 0;  // griddepcontrol.wait has returned in this warp
+        // Before its wait this warp only reads tables that the host wrote (descriptors, row pointers:
+        // their uploads are full stream dependencies), so the first tile's addresses are ready when
+        // the wait returns.  The rows are the caller's data: unless the caller has vouched that
+        // they were complete before this launch could start, the kernel before this one in the
+        // stream may be the one that writes them and may have triggered its dependents early, so
+        // the wait comes before the first copy.
+        bool late_fetch = R > 0;
+        bool waited = false;  // griddepcontrol.wait has returned in this warp
         long long rq0 = n_runs, rq1 = n_runs;  // the next two runs of this block
         auto fetch_run = [&]() -> long long {   // lane 0 asks, everybody gets the answer
             long long f = 0;
             if (lane == 0) f = G + (long long)atomicAdd(a.tile_counter, 1ull);
             return __shfl_sync(0xffffffffu, f, 0);
         };
-        if (R > 0 && !late_fetch) {
-            rq0 = fetch_run();
-            rq1 = fetch_run();
-        }
         // the tile after `tile` in this block's sequence (n_tiles when there is none); consumes a
         // prefetched run index at the end of a run
         auto next_tile = [&](long long tile) -> long long {
@@ -789,9 +784,10 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
             for (int ch = 0; ch < n_chunks; ++ch, ++item) {
                 const int st = item % nst;
                 const unsigned use = item / nst;
-                if (!waited && item >= nst) {
-                    // reusing a stage needs the consumers, and they start only after the previous
-                    // kernel: from here on this warp's bounded waits must not count its run time
+                if (!waited && (!a.early_rows || item >= nst)) {
+                    // the rows may not be read yet (default), or a stage is about to be reused, which
+                    // needs the consumers, and they start only after the previous kernel: from here on
+                    // this warp's bounded waits must not count that kernel's run time
                     griddep_wait();
                     trigger_early();
                     waited = true;
@@ -1166,7 +1162,15 @@ __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const _
     const long long n_tiles = a.n_tiles, G = gridDim.x;
     long long c = blockIdx.x;
     TileDesc d = {}, dn = {};
-    if (c < n_tiles) d = a.tiles[c];
+    // Before the wait: only tables that the host wrote (descriptor, the tensor's pointers and flags).
+    float *wq = nullptr, *vq = nullptr;
+    unsigned fl = 0;
+    if (c < n_tiles) {
+        d = a.tiles[c];
+        wq = (float *)a.wv[d.tensor];
+        vq = (float *)a.wv[T + d.tensor];
+        fl = a.wflags[d.tensor];
+    }
     griddep_wait();
     griddep_launch();
     // the counter belongs to the update launches; it is touched only after the wait, so that even
@@ -1180,10 +1184,10 @@ __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const _
         const long long nc = s_next[buf];
         if (tid == 0 && nc < n_tiles) s_next[buf ^ 1] = G + (long long)atomicAdd(a.next_chunk, 1ull);
         if (nc < n_tiles) dn = a.tiles[nc];
-        float *w = (float *)a.wv[d.tensor] + d.first;
-        float *v = (float *)a.wv[T + d.tensor] + d.first;
+        float *w = wq + d.first;
+        float *v = vq + d.first;
         const float *g = a.gbar + d.goff;
-        const bool vec = (a.wflags[d.tensor] & 1u) != 0;
+        const bool vec = (fl & 1u) != 0;
         const int len = d.len;
         if (vec && len == 1024 * C) {
             float4 gg[C], ww[C], vv[C];
@@ -1218,6 +1222,11 @@ __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const _
                 v[e] = vn;
                 w[e] = fmaf(-eta, vn, w[e]);
             }
+        }
+        if (nc < n_tiles && dn.tensor != d.tensor) {  // the next tile's tensor, requested before the barrier
+            wq = (float *)a.wv[dn.tensor];
+            vq = (float *)a.wv[T + dn.tensor];
+            fl = a.wflags[dn.tensor];
         }
         __syncthreads();
         c = nc;
