@@ -693,12 +693,14 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
         // the wait comes before the first copy.
         bool late_fetch = R > 0;
         bool waited = false;  // griddepcontrol.wait has returned in this warp
-        long long rq0 = n_runs, rq1 = n_runs;  // the next two runs of this block
-        auto fetch_run = [&]() -> long long {   // lane 0 asks, everybody gets the answer
-            long long f = 0;
-            if (lane == 0) f = G + (long long)atomicAdd(a.tile_counter, 1ull);
-            return __shfl_sync(0xffffffffu, f, 0);
+        // The next two runs of this block, known to all lanes, and a third that lane 0 has asked the
+        // counter for but not yet passed on: the answer is only looked at when the next run is
+        // taken, a whole run later, so the warp never waits for the atomic's round trip.
+        long long rq0 = n_runs, rq1 = n_runs, rq2_lane0 = n_runs;
+        auto ask_run = [&]() {   // lane 0 asks the counter; nobody waits
+            if (lane == 0) rq2_lane0 = G + (long long)atomicAdd(a.tile_counter, 1ull);
         };
+        auto take_asked = [&]() -> long long { return __shfl_sync(0xffffffffu, rq2_lane0, 0); };
         // the tile after `tile` in this block's sequence (n_tiles when there is none); consumes a
         // prefetched run index at the end of a run
         auto next_tile = [&](long long tile) -> long long {
@@ -707,7 +709,12 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
             if ((tile + 1) % R != 0 && tile + 1 < n_tiles) return tile + 1;
             const long long r = rq0;
             rq0 = rq1;
-            rq1 = (late_fetch || r >= n_runs) ? n_runs : fetch_run();
+            if (late_fetch || r >= n_runs) {
+                rq1 = n_runs;
+            } else {
+                rq1 = take_asked();
+                if (rq1 < n_runs) ask_run();
+            }
             return r < n_runs ? r * R : n_tiles;
         };
         TileDesc d0, d1 = {}, d2 = {};
@@ -831,8 +838,11 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                     trigger_early();
                     waited = true;
                 }
-                rq0 = fetch_run();
-                rq1 = fetch_run();
+                ask_run();
+                rq0 = take_asked();
+                ask_run();
+                rq1 = take_asked();
+                ask_run();
                 // the sequence was built without the counter: rebuild what follows this tile
                 t_next = next_tile(t);
                 t1_next = next_tile(t_next);
@@ -871,6 +881,10 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
         // the sums of the last tiles; with the static assignment, the block's one pair
         for (unsigned seq = q >= (unsigned)kSlots ? q - kSlots + 1 : 0u; R > 0 && seq < q && !timed_out; ++seq)
             if (!deliver(seq)) timed_out = true;
+        // The answer to the last question put to the counter must have arrived before this block
+        // takes its exit ticket: the block that finishes last resets the counter, and an increment
+        // still on its way would land after the reset.  (Looking at the value makes the warp wait.)
+        if (R > 0 && take_asked() < 0) timed_out = true;
         if (timed_out) atomicExch(&abort_flag, 1);
         // Every copy this warp has issued must have landed before the block may leave (its shared
         // memory is handed to the next block): wait for the last phase of each stage, with the long
