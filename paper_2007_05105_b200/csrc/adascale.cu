@@ -585,8 +585,7 @@ adascale_status do_update(adascale_ctx *ctx, void *const *params, void *const *m
     a.n_tiles = n_tiles;
     a.gbar = ctx->d_gbar;
     a.st = ctx->d_state;
-    a.next_chunk = reinterpret_cast<u64 *>(ctx->d_ticket + 64);
-    a.exit_ticket = ctx->d_ticket + 128;
+    a.next_tile = ctx->d_ticket + 64;
     a.T = T;
     a.rho = (float)ctx->rho;
     a.lambda = (float)ctx->lambda;
@@ -715,6 +714,10 @@ adascale_status adascale_init(const adascale_config *cfg, adascale_ctx **out)
     }
     ctx->gbar_elems = g;
     ctx->n_utiles = (long long)utiles.size();
+    if (ctx->n_utiles > 0xffffffffLL) {  // the update kernel's tile counter is 32 bits wide
+        delete ctx;
+        return ADASCALE_ERR_TOO_LARGE;
+    }
     ctx->rtiles_cap = rcap;
 
     DeviceGuard guard(ctx->device);

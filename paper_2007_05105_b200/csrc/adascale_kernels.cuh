@@ -148,8 +148,7 @@ struct UpdateArgs {
     long long n_tiles;
     const float *gbar;
     const DevState *st;
-    u64 *next_chunk;          // tiles handed out beyond each block's first; zero between launches
-    unsigned *exit_ticket;    // the block that leaves last resets both counters
+    unsigned *next_tile;      // tiles handed out beyond each block's first; wraps to zero by itself
     int T;
     float rho, lambda;
 };
@@ -1167,7 +1166,9 @@ __device__ __forceinline__ void update4(float4 &ww, float4 &vv, const float4 &gg
 // efficient), and no SM idles at the end.  The counter value is fetched one tile ahead and the
 // descriptor of the next tile while the current one is processed.  A tile is kUpdateTile =
 // 1024 * C elements: C 128-bit accesses per array and thread, all requested before the first
-// is used.  The block that leaves last resets the counters for the next launch.
+// is used.  The counter needs no reset: every block asks once more than it gets tiles (its last
+// answer is the one that tells it to stop), so a launch asks exactly n_tiles times, and the
+// counter is an atomicInc that wraps to zero after n_tiles increments.
 __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const __grid_constant__ UpdateArgs a)
 {
     constexpr int C = kUpdateVecs;
@@ -1187,16 +1188,20 @@ __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const _
     }
     griddep_wait();
     griddep_launch();
+    // a skipped iteration (non-finite sums, or a bounded wait that gave up) changes nothing; every
+    // block sees the same state, so either all of them ask the counter or none does
+    const bool skip = (a.st->status & ADASCALE_STATUS_NONFINITE) || a.st->fault;
+    if (skip) return;
+    const float eta = (float)a.st->eta;
     // the counter belongs to the update launches; it is touched only after the wait, so that even
     // two update launches in a row cannot meet on it
-    if (tid == 0) s_next[0] = G + (long long)atomicAdd(a.next_chunk, 1ull);
-    const bool skip = (a.st->status & ADASCALE_STATUS_NONFINITE) || a.st->fault;
-    const float eta = (float)a.st->eta;
+    const unsigned wrap = (unsigned)(n_tiles - 1);
+    if (tid == 0) s_next[0] = G + (long long)atomicInc(a.next_tile, wrap);
     __syncthreads();
     int buf = 0;
-    while (c < n_tiles && !skip) {
+    while (c < n_tiles) {
         const long long nc = s_next[buf];
-        if (tid == 0 && nc < n_tiles) s_next[buf ^ 1] = G + (long long)atomicAdd(a.next_chunk, 1ull);
+        if (tid == 0 && nc < n_tiles) s_next[buf ^ 1] = G + (long long)atomicInc(a.next_tile, wrap);
         if (nc < n_tiles) dn = a.tiles[nc];
         float *w = wq + d.first;
         float *v = vq + d.first;
@@ -1246,13 +1251,6 @@ __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const _
         c = nc;
         buf ^= 1;
         d = dn;
-    }
-    if (tid == 0) {
-        __threadfence();
-        if (atomicAdd(a.exit_ticket, 1u) == gridDim.x - 1) {
-            *a.next_chunk = 0ull;
-            *a.exit_ticket = 0u;
-        }
     }
 }
 
