@@ -735,7 +735,7 @@ adascale_status adascale_init(const adascale_config *cfg, adascale_ctx **out)
         CU(cudaMalloc(&ctx->d_partials, (size_t)(ctx->sms * kReduceBlocksPerSM + 1) * sizeof(double2)));
         CU(cudaMalloc(&ctx->d_run_partials,
                       (size_t)(rcap + ctx->sms * kReduceBlocksPerSM + 1) * sizeof(double2)));
-        CU(cudaMalloc(&ctx->d_ticket, 4 * 256));  // four counters, 256 bytes apart
+        CU(cudaMalloc(&ctx->d_ticket, 4 * 256));  // counters, 256 bytes apart: exit ticket, update tiles, (spare), runs
         CU(cudaMemset(ctx->d_ticket, 0, 4 * 256));
         CU(cudaMalloc(&ctx->d_state, sizeof(DevState)));
         CU(cudaMemset(ctx->d_state, 0, sizeof(DevState)));
