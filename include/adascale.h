@@ -240,6 +240,17 @@ adascale_status adascale_set_scale(adascale_ctx *ctx, int32_t S);
 adascale_status adascale_set_wait_limit(adascale_ctx *ctx, uint32_t polls);
 
 /*
+ * How the reduce kernel hands its tiles to the blocks, for the following steps: run_tiles = -1
+ * (default) lets the library choose by the job's size (see adascale_tiling); 0 assigns tile t to
+ * block t mod grid; 1 .. 64 hands out runs of that many consecutive tiles from a device
+ * counter.  Every setting gives sums that are reproducible from run to run; different settings
+ * add the same terms in different orders and so may differ in the last bits.  It exists for
+ * tests (so that small jobs can exercise the path of large ones) and for tuning.  No counterpart
+ * in the paper.  Errors: INVALID_ARG.
+ */
+adascale_status adascale_set_tile_runs(adascale_ctx *ctx, int32_t run_tiles);
+
+/*
  * Checkpoint / resume of the scalar state (tau, averages, counters): buf is a host
  * buffer of ADASCALE_STATE_BYTES.  Both calls wait for the device.  set_state rejects a
  * buffer that get_state did not write (INVALID_ARG).  No counterpart in the paper.

@@ -22,7 +22,7 @@ STATE_BYTES = 128
 
 EXPORTS = ("adascale_init", "adascale_step", "adascale_reduce", "adascale_update", "adascale_reduce_sums",
            "adascale_apply_sums", "adascale_get_gain_tau",
-           "adascale_mean_grad", "adascale_set_scale", "adascale_set_wait_limit", "adascale_get_state", "adascale_set_state",
+           "adascale_mean_grad", "adascale_set_scale", "adascale_set_wait_limit", "adascale_set_tile_runs", "adascale_get_state", "adascale_set_state",
            "adascale_step_host", "adascale_stream_probe", "adascale_tiling", "adascale_grad_stats_static", "adascale_launch_count",
            "adascale_destroy",
            "adascale_strerror", "adascale_last_error")
@@ -72,6 +72,7 @@ def _load(path=LIB_PATH):
     L.adascale_mean_grad.argtypes = [vp, vpp]
     L.adascale_set_scale.argtypes = [vp, C.c_int32]
     L.adascale_set_wait_limit.argtypes = [vp, C.c_uint32]
+    L.adascale_set_tile_runs.argtypes = [vp, C.c_int32]
     L.adascale_get_state.argtypes = [vp, vp]
     L.adascale_set_state.argtypes = [vp, vp]
     L.adascale_step_host.argtypes = [vp, vpp, vpp, vpp, C.POINTER(LrSchedule), C.POINTER(Stats), vp]
@@ -242,6 +243,10 @@ class AdaScale:
     def set_wait_limit(self, polls):
         """Bound of the reduce kernel's handshake waits (a test hook for the give-up path)."""
         self._check(lib.adascale_set_wait_limit(self._ctx, int(polls)))
+
+    def set_tile_runs(self, run_tiles):
+        """-1: the library chooses; 0: static assignment; n: runs of n tiles from the device counter."""
+        self._check(lib.adascale_set_tile_runs(self._ctx, int(run_tiles)))
 
     def get_state(self) -> bytes:
         buf = C.create_string_buffer(STATE_BYTES)

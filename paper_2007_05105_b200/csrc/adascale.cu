@@ -183,6 +183,7 @@ struct adascale_ctx {
     cudaStream_t last_stream = nullptr;
     bool reduced = false;
     unsigned wait_spins = kSpinLimit;  // bound of the reduce kernel's handshake waits
+    int forced_runs = -1;              // >= 0: tiles per run (0 = static assignment) whatever the job's size
     long long launches = 0;
     void *d_stage = nullptr;     // host-gradient staging (adascale_step_host)
     std::vector<const void *> stage_ptrs;
@@ -516,7 +517,7 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
     a.lambda = (float)ctx->lambda;
     a.partials = ctx->d_partials;
     a.run_partials = ctx->d_run_partials;
-    a.run_tiles = run_tiles_for(n_tiles, S);
+    a.run_tiles = ctx->forced_runs >= 0 ? ctx->forced_runs : run_tiles_for(n_tiles, S);
     // Two stages in flight per block are enough and measured 2-5 % faster than three when tiles are
     // assigned statically; with runs from a counter three were 2 % faster.
     a.stages = a.run_tiles > 0 ? (unsigned)kStages : 2u;
@@ -926,6 +927,13 @@ adascale_status adascale_set_wait_limit(adascale_ctx *ctx, uint32_t polls)
 {
     if (!ctx) return ADASCALE_ERR_INVALID_ARG;
     ctx->wait_spins = polls;
+    return ADASCALE_OK;
+}
+
+adascale_status adascale_set_tile_runs(adascale_ctx *ctx, int32_t run_tiles)
+{
+    if (!ctx || run_tiles < -1 || run_tiles > 64) return ADASCALE_ERR_INVALID_ARG;
+    ctx->forced_runs = run_tiles;
     return ADASCALE_OK;
 }
 

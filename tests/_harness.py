@@ -103,11 +103,13 @@ class Pair:
     """
 
     def __init__(self, numels, S, grad_dtype="f32", momentum=0.0, weight_decay=0.0, eps=1e-6, theta=-1.0,
-                 flags=0, max_S=0, lr=None):
+                 flags=0, max_S=0, lr=None, tile_runs=-1):
         self.numels = list(numels)
         self.S = S
         self.lr_spec = lr or {"kind": "const", "eta0": 0.1}
         self.dev = B.AdaScale(numels, S, grad_dtype, momentum, weight_decay, eps, theta, flags, 0, max_S)
+        if tile_runs >= 0:  # small jobs can take the tile hand-out of large ones
+            self.dev.set_tile_runs(tile_runs)
         # the one-pass kernel is a device-side arrangement of the lagged mode: same oracle
         self.fused = bool(flags & B.FLAG_FUSED)
         self.orc = oracle.Oracle(S, momentum, weight_decay, eps, theta, flags & ~B.FLAG_FUSED, nthreads=NTHREADS)

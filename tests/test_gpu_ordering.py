@@ -25,11 +25,12 @@ DEV = torch.device("cuda:0")
 FUSED = B.FLAG_LAGGED | B.FLAG_FUSED
 
 
-def _run(wl, src, grads, w0, v0, steps, flags, sync_every_launch):
+def _run(wl, src, grads, w0, v0, steps, flags, sync_every_launch, tile_runs=-1):
     """`steps` iterations on fixed gradient buffers; returns (w, v, stats) as host arrays."""
     w, v = w0.clone(), v0.clone()
     wv, vv = src.views(w), src.views(v)
     ada = B.AdaScale(src.numels, wl.S, wl.grad_dtype, momentum=wl.momentum, weight_decay=wl.weight_decay, flags=flags)
+    ada.set_tile_runs(tile_runs)
     sched = H.device_lr(wl.lr)
     gp, wp, vp = B.pointer_array(grads), B.pointer_array(wv), B.pointer_array(vv)
     stream = torch.cuda.current_stream(DEV).cuda_stream
@@ -101,6 +102,27 @@ def test_back_to_back_steps_equal_synchronised_steps(name, steps, flags):
         assert (err_v <= tol_v).all(), "tensor %d momentum: worst %g x tolerance" % (k, float((err_v / tol_v).max()))
 
 
+@pytest.mark.parametrize("flags", [0, B.FLAG_GRADS_READY, FUSED, FUSED | B.FLAG_GRADS_READY],
+                         ids=["default", "grads_ready", "fused", "fused_grads_ready"])
+@pytest.mark.parametrize("runs", [1, 4])
+def test_back_to_back_steps_with_runs_from_the_counter(runs, flags):
+    """The same requirement with the tile hand-out of large jobs forced on resnet18: the run counter is
+    shared by consecutive launches, so a launch that touched it too early would process tiles twice."""
+    wl = synthetic.workload("resnet18")
+    wl.lr = {"kind": "const", "eta0": 0.01}
+    src = synthetic.GradientSource(wl, device=DEV)
+    grads = src.fill(0)
+    w0, v0 = src.init_params()
+    w_a, v_a, st_a = _run(wl, src, grads, w0, v0, 200, flags, False, runs)
+    w_b, v_b, st_b = _run(wl, src, grads, w0, v0, 200, flags, True, runs)
+    assert st_a.t == 200 and st_a.status_bits == 0 and st_a.tau == st_b.tau
+    assert np.array_equal(w_a.view(np.uint32), w_b.view(np.uint32))
+    assert np.array_equal(v_a.view(np.uint32), v_b.view(np.uint32))
+    w_c, v_c, st_c = _run(wl, src, grads, w0, v0, 200, flags, True, 0)        # static assignment
+    assert st_a.tau == pytest.approx(st_c.tau, rel=1e-12)
+    np.testing.assert_allclose(w_a, w_c, rtol=1e-5, atol=1e-7)
+
+
 def test_update_tiles_one_per_block_back_to_back():
     """A job with fewer update tiles than blocks: every block's only tile is its prefetched first tile."""
     wl = synthetic.workload("single_1m")
@@ -130,8 +152,9 @@ def _small_job(flags=0):
     return numels, S, rows, w, v
 
 
+@pytest.mark.parametrize("runs", [-1, 2])
 @pytest.mark.parametrize("polls", [0, 1])
-def test_a_wait_that_runs_out_is_reported_and_changes_nothing(polls):
+def test_a_wait_that_runs_out_is_reported_and_changes_nothing(polls, runs):
     """The handshake waits of the reduce kernel are given a limit that cannot (0 polls) or can hardly
     (1 poll) be met.  The step must return, report the condition, leave w and v alone, and keep
     skipping; a fresh context on the same device then passes a parity step."""
@@ -140,6 +163,7 @@ def test_a_wait_that_runs_out_is_reported_and_changes_nothing(polls):
     v_before = [t.clone() for t in v]
     ada = B.AdaScale(numels, S, "f32", momentum=0.9, weight_decay=1e-3)
     sched = B.make_schedule("const", eta0=0.1)
+    ada.set_tile_runs(runs)
     ada.set_wait_limit(polls)
     ada.step(rows, w, v, sched)
     st = ada.get_gain_tau(True)

@@ -89,6 +89,43 @@ def test_ragged_tensor_list(S, dtype):
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("runs", [1, 3, 8])
+@pytest.mark.parametrize("S", [2, 8, 9, 16, 33])
+def test_ragged_tensor_list_with_runs_from_the_counter(S, runs, dtype):
+    """The tile hand-out of large jobs (runs of tiles from a device counter, sums added up by the
+    producer warp), forced on a small ragged job plus one tensor of many tiles."""
+    gen = _gen(2000 + 10 * S + runs)
+    numels = RAGGED + [300000]
+    name = "bf16" if dtype == torch.bfloat16 else "f32"
+    pair = H.Pair(numels, S, name, momentum=0.9, weight_decay=1e-3, lr={"kind": "const", "eta0": 0.05}, tile_runs=runs)
+    w, v = _params(numels, gen)
+    pair.attach(w, v)
+    for step in range(2):
+        pair.step(_make_rows(numels, S, dtype, gen, k=[0.5, 10.0][step]), "S=%d runs=%d %s step %d" % (S, runs, name, step))
+    pair.close()
+
+
+def test_runs_from_the_counter_give_reproducible_sums_close_to_the_static_ones():
+    gen = _gen(2100)
+    numels = [200000, 4097, 77, 150016]
+    rows = _make_rows(numels, 16, torch.float32, gen)
+    w, v = _params(numels, gen)
+    seen = {}
+    for runs in (0, 1, 4, 4):
+        ada = B.AdaScale(numels, 16, "f32", momentum=0.9)
+        ada.set_tile_runs(runs)
+        for _ in range(3):
+            ada.reduce(rows, B.make_schedule())
+        st = ada.get_gain_tau(True)
+        seen.setdefault(runs, []).append((st.dev_sqsum, st.gbar_sqnorm, st.r))
+        ada.close()
+    assert seen[4][0] == seen[4][1]                       # bitwise, launch after launch and context after context
+    for runs in (1, 4):                                     # other orders of the same terms: last bits only
+        for a, b in zip(seen[runs][0], seen[0][0]):
+            assert a == pytest.approx(b, rel=1e-13)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
 @pytest.mark.parametrize("misalign", [1, 2, 3])
 def test_misaligned_pointers_take_the_scalar_path(misalign, dtype):
     gen = _gen(77 + misalign)
@@ -384,6 +421,20 @@ def test_fused_mode_against_the_lagged_oracle(S, dtype):
         st, _ = pair.step(rows, "fused S=%d %s step %d" % (S, name, step))
     if S > 1:
         assert st.r > 1.0  # the gain follows the averages from the second step on
+    pair.close()
+
+
+@pytest.mark.parametrize("runs", [1, 4])
+@pytest.mark.parametrize("S", [3, 16, 40])
+def test_fused_mode_with_runs_from_the_counter(S, runs):
+    gen = _gen(4150 + S + runs)
+    numels = RAGGED + [250000]
+    pair = H.Pair(numels, S, "bf16", momentum=0.9, weight_decay=1e-3, flags=FUSED, lr={"kind": "const", "eta0": 0.05},
+                  tile_runs=runs)
+    w, v = _params(numels, gen)
+    pair.attach(w, v)
+    for step in range(3):
+        pair.step(_make_rows(numels, S, torch.bfloat16, gen, k=1.0 + step), "fused S=%d runs=%d step %d" % (S, runs, step))
     pair.close()
 
 
