@@ -285,11 +285,11 @@ adascale_status adascale_stream_probe(int32_t kind, void *a, void *b, int64_t n_
  * (NULL = all aligned); n_blocks: grid size the tiling is tuned for.  Writes the number of
  * staged tiles before each tensor into tprefix[0..n_tensors] and of scalar-path tiles into
  * sprefix[0..n_tensors], the columns of one staged tile into *tile_cols and the rows of one
- * shared-memory stage into *rows.  With fewer than 32768 staged tiles, tile t is processed by
- * block t mod gridDim; larger jobs hand runs of 2 or 4 consecutive tiles to the blocks as they
- * become free, and the sums are added up per run and then over the runs in index order, so
- * the result does not depend on which block processed which run.  Makes no CUDA call.
- * Errors: INVALID_ARG.
+ * shared-memory stage into *rows.  With fewer than 32768 staged tiles, or S <= 8, tile t is
+ * processed by block t mod gridDim; larger jobs hand runs of 2 or 4 consecutive tiles to the
+ * blocks as they become free, and the sums are added up per run and then over the runs in
+ * index order, so the result does not depend on which block processed which run (see
+ * adascale_set_tile_runs).  Makes no CUDA call.  Errors: INVALID_ARG.
  */
 adascale_status adascale_tiling(const int64_t *numel, int32_t n_tensors, int32_t grad_dtype, int32_t S,
                                 const uint8_t *aligned, int32_t n_blocks, int64_t *tprefix, int64_t *sprefix,

@@ -4,17 +4,20 @@
 // Two kernels make up one iteration (paper: Sec. 3.2, App. B.3, Eq. 2-3):
 //   reduce  - streams the S x P gradient matrix once through shared memory (bulk asynchronous
 //             copies completed on mbarriers, a producer warp and eight consumer warps), writes
-//             the mean gradient and one pair (sum of squared deviations, squared norm of the
-//             mean) per block; the block that finishes last adds the pairs in index order and
-//             runs the scalar part (estimates, clamps, moving averages, r_t, eta_t, tau_{t+1}).
+//             the mean gradient and pairs (sum of squared deviations, squared norm of the mean)
+//             per block or per run of tiles; the block that finishes last adds the pairs in
+//             index order and runs the scalar part (estimates, clamps, moving averages, r_t,
+//             eta_t, tau_{t+1}).
 //   update  - v <- rho v + (gbar + lambda w), w <- w - eta_t v, reading eta_t from the device.
 // Three trivial streaming kernels calibrate the bandwidth ceiling.
 // The path is bound by HBM bandwidth; there is no contraction, hence no tensor-core work.
 //
-// Work distribution: every tensor is cut into tiles; tile t belongs to block t mod gridDim.
-// All blocks therefore advance through each gradient row as one front, which keeps DRAM
-// pages hot, and the split does not depend on how the hardware schedules blocks, so the
-// fixed-order sums are reproducible from run to run.
+// Work distribution: every tensor is cut into tiles.  Small jobs: tile t belongs to block
+// t mod gridDim.  Large jobs: runs of consecutive tiles (reduce) or single tiles (update) are
+// handed to the blocks from a device counter as they become free.  Either way all blocks
+// advance through each array as one narrow front, which keeps DRAM pages hot, and the sums are
+// added up in an order that does not depend on how the hardware schedules blocks, so they are
+// reproducible from run to run.
 #include "../../include/adascale.h"
 
 #include <cuda_runtime.h>
@@ -86,8 +89,8 @@ struct Sched {
 };
 
 // One tile of work: `len` elements of tensor `tensor` starting at element `first`; `goff` is
-// where the tile's mean gradient lives in the library's workspace.  Tile t belongs to block
-// t mod gridDim.  The descriptors hold no pointers, so they change only with the tiling.
+// where the tile's mean gradient lives in the library's workspace.  The descriptors hold no
+// pointers, so they change only with the tiling.
 struct __align__(16) TileDesc {
     long long first;
     long long goff;
