@@ -491,17 +491,65 @@ template <int CPT> struct PairLoad<ADASCALE_BF16, CPT> {
     }
 };
 
+// CPT bf16 columns of one staged row as CPT/2 raw 32-bit words (two elements each).
+template <int CPT, int OFF>
+__device__ __forceinline__ void load_words(unsigned addr, unsigned *u)
+{
+    if constexpr (CPT == 4)
+        asm volatile("ld.shared.v2.b32 {%0, %1}, [%2+%3];" : "=r"(u[0]), "=r"(u[1]) : "r"(addr), "n"(OFF));
+    else
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4+%5];"
+                     : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3])
+                     : "r"(addr), "n"(OFF));
+}
+// Median of three, on both bf16 elements of a word at once.  The median of three bf16 values is
+// one of them, so taking it before widening is exact; like fminf / fmaxf, the packed min / max
+// return the other operand when one is NaN.
+__device__ __forceinline__ unsigned median3_bf16x2(unsigned a, unsigned b, unsigned e)
+{
+    unsigned r;
+    asm("{\n\t.reg .b32 lo, hi, t;\n\t"
+        "min.bf16x2 lo, %1, %2;\n\tmax.bf16x2 hi, %1, %2;\n\t"
+        "min.bf16x2 t, hi, %3;\n\tmax.bf16x2 %0, lo, t;\n\t}"
+        : "=r"(r)
+        : "r"(a), "r"(b), "r"(e));
+    return r;
+}
+// x - c for the two bf16 elements of one 32-bit word.  sm_100 subtracts an fp32 from a bf16
+// operand in one instruction (the operand is widened exactly, the difference rounded once: the
+// same result as widening first), so no shift or mask is spent per element.
+__device__ __forceinline__ f2 sub2_bf16(unsigned u, f2 c)
+{
+    f2 r;
+    asm("{\n\t.reg .b16 xl, xh;\n\t.reg .f32 cl, ch, dl, dh;\n\t"
+        "mov.b32 {xl, xh}, %1;\n\tmov.b64 {cl, ch}, %2;\n\t"
+        "sub.rn.f32.bf16 dl, xl, cl;\n\tsub.rn.f32.bf16 dh, xh, ch;\n\t"
+        "mov.b64 %0, {dl, dh};\n\t}"
+        : "=l"(r)
+        : "r"(u), "l"(c));
+    return r;
+}
+
 // One staged row into the running sums: d = x - c, p1 += d, s2 += d * d.
 template <int DT, int CPT, int OFF>
 __device__ __forceinline__ void consume_row(unsigned addr, const f2 *c, f2 *p1, f2 *s2)
 {
-    f2 x[CPT / 2];
-    PairLoad<DT, CPT>::template load<OFF>(addr, x);
+    f2 d[CPT / 2];
+    if constexpr (DT == ADASCALE_BF16) {
+        unsigned u[CPT / 2];
+        load_words<CPT, OFF>(addr, u);
+#pragma unroll
+        for (int j = 0; j < CPT / 2; ++j) d[j] = sub2_bf16(u[j], c[j]);
+    } else {
+        f2 x[CPT / 2];
+        PairLoad<DT, CPT>::template load<OFF>(addr, x);
+#pragma unroll
+        for (int j = 0; j < CPT / 2; ++j) d[j] = sub2(x[j], c[j]);
+    }
 #pragma unroll
     for (int j = 0; j < CPT / 2; ++j) {
-        const f2 d = sub2(x[j], c[j]);
-        p1[j] = add2(p1[j], d);
-        s2[j] = fma2(d, d, s2[j]);
+        p1[j] = add2(p1[j], d[j]);
+        s2[j] = fma2(d[j], d[j], s2[j]);
     }
 }
 
@@ -956,7 +1004,16 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                 unsigned addr = lane_base + (unsigned)st * stage_bytes;
                 if (active) {
                     if (ch == 0) {
-                        if (S >= 3) {  // shift = median of the first three rows
+                        if (DT == ADASCALE_BF16 && S >= 3) {  // the same median, taken on the raw words
+                            if constexpr (DT == ADASCALE_BF16) {
+                                unsigned u0[NP], u1[NP], u2[NP];
+                                load_words<CPT, 0>(addr, u0);
+                                load_words<CPT, kRowBytes>(addr, u1);
+                                load_words<CPT, 2 * kRowBytes>(addr, u2);
+#pragma unroll
+                                for (int j = 0; j < NP; ++j) c[j] = widen2(median3_bf16x2(u0[j], u1[j], u2[j]));
+                            }
+                        } else if (S >= 3) {  // shift = median of the first three rows
                             f2 x0[NP], x1[NP], x2[NP];
                             PairLoad<DT, CPT>::template load<0>(addr, x0);
                             PairLoad<DT, CPT>::template load<kRowBytes>(addr, x1);
