@@ -57,6 +57,7 @@ constexpr int kMaxS = 4096;
 constexpr unsigned kSpinLimit = 1u << 22; // bounded waits: give up, flag, leave (default of the handshake waits,
                                           // fixed bound of the wait for copies that are already in flight)
 constexpr unsigned long long kWaitNs = 2000000000ull;  // and no wait lasts longer than two seconds
+constexpr unsigned kWaitHintNs = 20000;   // how long one poll of a barrier may sleep (it wakes on completion)
 
 typedef unsigned long long u64;
 
@@ -378,16 +379,18 @@ __device__ __forceinline__ u64 global_ns()
 }
 // Returns false if the phase did not complete within `limit` polls or within kWaitNs of wall
 // time, whichever comes first (one poll can itself suspend the thread for a while, so a poll
-// count alone does not bound the time).
+// count alone does not bound the time).  Each poll may sleep up to kWaitHintNs and wakes when
+// the phase completes: with the default (much shorter) sleep a third of all instructions the
+// reduce kernel issued were polls of waiting warps, and it ran 0.4 % slower.
 __device__ __forceinline__ bool mbar_wait(u64 *bar, unsigned parity, unsigned limit)
 {
     const unsigned addr = smem_u32(bar);
     u64 t0 = 0;
     for (unsigned spin = 0; spin < limit; ++spin) {
         unsigned done;
-        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
                      : "=r"(done)
-                     : "r"(addr), "r"(parity)
+                     : "r"(addr), "r"(parity), "r"(kWaitHintNs)
                      : "memory");
         if (done) return true;
         if ((spin & 63u) == 63u) {
