@@ -494,6 +494,10 @@ template <int CPT> struct PairLoad<ADASCALE_BF16, CPT> {
     }
 };
 
+// What a thread holds of two adjacent columns of a row before the shift is subtracted.
+template <int DT> struct Held { typedef f2 type; };                       // fp32: the packed pair
+template <> struct Held<ADASCALE_BF16> { typedef unsigned type; };       // bf16: the raw word
+
 // CPT bf16 columns of one staged row as CPT/2 raw 32-bit words (two elements each).
 template <int CPT, int OFF>
 __device__ __forceinline__ void load_words(unsigned addr, unsigned *u)
@@ -531,6 +535,20 @@ __device__ __forceinline__ f2 sub2_bf16(unsigned u, f2 c)
         : "=l"(r)
         : "r"(u), "l"(c));
     return r;
+}
+
+// A row that is already in registers (raw words for bf16, packed pairs for fp32) into the running sums.
+template <int DT, int CPT>
+__device__ __forceinline__ void consume_held(const typename Held<DT>::type *x, const f2 *c, f2 *p1, f2 *s2)
+{
+#pragma unroll
+    for (int j = 0; j < CPT / 2; ++j) {
+        f2 d;
+        if constexpr (DT == ADASCALE_BF16) d = sub2_bf16(x[j], c[j]);
+        else d = sub2(x[j], c[j]);
+        p1[j] = add2(p1[j], d);
+        s2[j] = fma2(d, d, s2[j]);
+    }
 }
 
 // One staged row into the running sums: d = x - c, p1 += d, s2 += d * d.
@@ -1006,38 +1024,53 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                 const int rows = S - r0 < rps ? S - r0 : rps;
                 unsigned addr = lane_base + (unsigned)st * stage_bytes;
                 if (active) {
+                    int r = 0;
                     if (ch == 0) {
-                        if (DT == ADASCALE_BF16 && S >= 3) {  // the same median, taken on the raw words
-                            if constexpr (DT == ADASCALE_BF16) {
-                                unsigned u0[NP], u1[NP], u2[NP];
-                                load_words<CPT, 0>(addr, u0);
-                                load_words<CPT, kRowBytes>(addr, u1);
-                                load_words<CPT, 2 * kRowBytes>(addr, u2);
 #pragma unroll
-                                for (int j = 0; j < NP; ++j) c[j] = widen2(median3_bf16x2(u0[j], u1[j], u2[j]));
+                        for (int j = 0; j < NP; ++j) s1[j] = s2[j] = 0ull;  // +0.0f, +0.0f
+                        if (S >= 3) {  // shift = median of the first three rows
+                            typename Held<DT>::type x0[NP], x1[NP], x2[NP];
+                            if constexpr (DT == ADASCALE_BF16) {  // taken on the raw words, widened once
+                                load_words<CPT, 0>(addr, x0);
+                                load_words<CPT, kRowBytes>(addr, x1);
+                                load_words<CPT, 2 * kRowBytes>(addr, x2);
+#pragma unroll
+                                for (int j = 0; j < NP; ++j) c[j] = widen2(median3_bf16x2(x0[j], x1[j], x2[j]));
+                            } else {
+                                PairLoad<DT, CPT>::template load<0>(addr, x0);
+                                PairLoad<DT, CPT>::template load<kRowBytes>(addr, x1);
+                                PairLoad<DT, CPT>::template load<2 * kRowBytes>(addr, x2);
+#pragma unroll
+                                for (int j = 0; j < NP; ++j) {
+                                    float a0, a1, b0, b1, e0, e1;
+                                    unpack2(x0[j], a0, a1);
+                                    unpack2(x1[j], b0, b1);
+                                    unpack2(x2[j], e0, e1);
+                                    const float m0 = fmaxf(fminf(a0, b0), fminf(fmaxf(a0, b0), e0));
+                                    const float m1 = fmaxf(fminf(a1, b1), fminf(fmaxf(a1, b1), e1));
+                                    c[j] = pack2(m0, m1);
+                                }
                             }
-                        } else if (S >= 3) {  // shift = median of the first three rows
-                            f2 x0[NP], x1[NP], x2[NP];
-                            PairLoad<DT, CPT>::template load<0>(addr, x0);
-                            PairLoad<DT, CPT>::template load<kRowBytes>(addr, x1);
-                            PairLoad<DT, CPT>::template load<2 * kRowBytes>(addr, x2);
+                            if (rows >= 8) {  // first block of 8: the three rows are still in registers
 #pragma unroll
-                            for (int j = 0; j < NP; ++j) {
-                                float a0, a1, b0, b1, e0, e1;
-                                unpack2(x0[j], a0, a1);
-                                unpack2(x1[j], b0, b1);
-                                unpack2(x2[j], e0, e1);
-                                const float m0 = fmaxf(fminf(a0, b0), fminf(fmaxf(a0, b0), e0));
-                                const float m1 = fmaxf(fminf(a1, b1), fminf(fmaxf(a1, b1), e1));
-                                c[j] = pack2(m0, m1);
+                                for (int j = 0; j < NP; ++j) p1[j] = 0ull;
+                                consume_held<DT, CPT>(x0, c, p1, s2);
+                                consume_held<DT, CPT>(x1, c, p1, s2);
+                                consume_held<DT, CPT>(x2, c, p1, s2);
+                                consume_row<DT, CPT, 3 * kRowBytes>(addr, c, p1, s2);
+                                consume_row<DT, CPT, 4 * kRowBytes>(addr, c, p1, s2);
+                                consume_row<DT, CPT, 5 * kRowBytes>(addr, c, p1, s2);
+                                consume_row<DT, CPT, 6 * kRowBytes>(addr, c, p1, s2);
+                                consume_row<DT, CPT, 7 * kRowBytes>(addr, c, p1, s2);
+#pragma unroll
+                                for (int j = 0; j < NP; ++j) s1[j] = add2(s1[j], p1[j]);
+                                addr += 8 * kRowBytes;
+                                r = 8;
                             }
                         } else {
                             PairLoad<DT, CPT>::template load<0>(addr, c);
                         }
-#pragma unroll
-                        for (int j = 0; j < NP; ++j) s1[j] = s2[j] = 0ull;  // +0.0f, +0.0f
                     }
-                    int r = 0;
                     for (; r + 8 <= rows; r += 8) {  // s1 in blocks of 8 rows
 #pragma unroll
                         for (int j = 0; j < NP; ++j) p1[j] = 0ull;
