@@ -176,13 +176,21 @@ adascale_status adascale_step(adascale_ctx *ctx, const void *const *grads, void 
  * forms sum_i ||g_i - gbar||^2 and ||gbar||^2 and runs the scalar part (estimates,
  * averages, r_t, eta_t, tau_{t+1}) on the device (Sec. 3.2, App. B.3, Eq. 3).
  * Arguments as in adascale_step.  One kernel launch.
+ * Where the scalar part runs is the library's business: for jobs whose tiles are assigned
+ * statically (see adascale_tiling) the reduce kernel stops at one pair of sums per block
+ * and the kernel that follows completes the iteration - the update kernel of
+ * adascale_update / adascale_step, each of whose blocks adds up the pairs itself, or, when
+ * adascale_get_gain_tau, adascale_get_state, adascale_apply_sums or another adascale_reduce
+ * comes first, a one-block kernel that the library enqueues before serving that call (one
+ * more launch in adascale_launch_count).  The state a caller reads is the same either way.
  */
 adascale_status adascale_reduce(adascale_ctx *ctx, const void *const *grads,
                                 const adascale_lr_schedule *sched, void *cuda_stream);
 
 /*
  * Second half: v <- rho v + (gbar + lambda w); w <- w - eta_t v with the eta_t that the
- * preceding adascale_reduce left on the device (Eq. 2, Sec. 3.4).  ERR_STATE if no
+ * preceding adascale_reduce left on the device (Eq. 2, Sec. 3.4), or that this kernel
+ * completes itself where the reduce launch left the scalar part open.  ERR_STATE if no
  * reduce precedes it.  One kernel launch.
  */
 adascale_status adascale_update(adascale_ctx *ctx, void *const *params, void *const *momentum,

@@ -174,6 +174,13 @@ struct adascale_ctx {
     double2 *d_run_partials = nullptr;    // per run of staged tiles, or per block
     unsigned *d_ticket = nullptr;
     DevState *d_state = nullptr;
+    // A reduce launch of a small or mid-size job leaves the scalar part of its iteration to the
+    // kernel that follows: normally the update, else a one-block kernel enqueued as soon as
+    // anything else needs the state.
+    bool scalar_open = false;
+    int open_pairs = 0;
+    ScalarCfg open_sc;
+    Sched open_sched;
     PtrTable tg, tw;
     long long n_tiles = 0, n_stiles = 0;  // of the descriptors on the device
     DevState *h_snap = nullptr;  // pinned
@@ -492,10 +499,33 @@ long long run_tiles_for(long long n_tiles, int S)
     return n_tiles >= 4 * kDynamicMinTiles ? 4 : 2;
 }
 
+// Completes an iteration whose scalar part a reduce launch has left open and that no update launch took over.
+adascale_status finish_open_scalar(adascale_ctx *ctx, cudaStream_t s)
+{
+    if (!ctx->scalar_open) return ADASCALE_OK;
+    FinishArgs a;
+    a.st = ctx->d_state;
+    a.partials = ctx->d_partials;
+    a.n_partials = ctx->open_pairs;
+    a.snapshot = reinterpret_cast<const RawState *>(ctx->d_ticket + 128);
+    a.sc = ctx->open_sc;
+    a.sched = ctx->open_sched;
+    cudaError_t e = launch_overlapped(k_finish, 1, kThreads, 0, s, a);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "launch of the scalar kernel");
+    ctx->launches += 1;
+    ctx->scalar_open = false;
+    ctx->last_stream = s;
+    return ADASCALE_OK;
+}
+
 adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const adascale_lr_schedule *sched,
                           cudaStream_t s, bool fused, double *sums_out = nullptr)
 {
     const int S = ctx->S, T = ctx->T;
+    if (ctx->scalar_open) {  // two reduce launches in a row: the first one's iteration is completed first
+        adascale_status so = finish_open_scalar(ctx, s);
+        if (so != ADASCALE_OK) return so;
+    }
     const size_t esz = ctx->dtype == ADASCALE_BF16 ? 2 : 4;
     const int max_blocks = ctx->sms * kReduceBlocksPerSM;
     adascale_status st = sync_reduce_table(ctx, grads, s);
@@ -525,6 +555,10 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
     a.tile_counter = reinterpret_cast<u64 *>(ctx->d_ticket + 192);
     a.st = ctx->d_state;
     a.sums_out = sums_out;
+    // Static assignment, two-kernel form, sums not wanted by the caller: one pair per block is all
+    // that is left to add up, and every block of the update kernel can do that itself.
+    const bool leave_open = !fused && !sums_out && a.run_tiles == 0;
+    a.snapshot = leave_open ? reinterpret_cast<RawState *>(ctx->d_ticket + 128) : nullptr;
     a.spin_limit = ctx->wait_spins;
     a.early_rows = (ctx->flags & ADASCALE_FLAG_GRADS_READY) ? 1u : 0u;
     a.S = S;
@@ -541,6 +575,12 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
     ctx->launches += 1;
     ctx->reduced = true;
     ctx->last_stream = s;
+    if (leave_open) {
+        ctx->scalar_open = true;
+        ctx->open_pairs = (int)nb;
+        ctx->open_sc = a.sc;
+        ctx->open_sched = a.sched;
+    }
     return ADASCALE_OK;
 }
 
@@ -590,10 +630,17 @@ adascale_status do_update(adascale_ctx *ctx, void *const *params, void *const *m
     a.T = T;
     a.rho = (float)ctx->rho;
     a.lambda = (float)ctx->lambda;
+    a.partials = ctx->d_partials;
+    a.n_partials = ctx->open_pairs;
+    a.snapshot = reinterpret_cast<const RawState *>(ctx->d_ticket + 128);
+    a.sc = ctx->open_sc;
+    a.sched = ctx->open_sched;
     long long nb = n_tiles;
     if (nb > (long long)ctx->sms * kUpdateBlocksPerSM) nb = (long long)ctx->sms * kUpdateBlocksPerSM;
-    cudaError_t e = launch_overlapped(k_update, (int)nb, kThreads, 0, s, a);
+    cudaError_t e = ctx->scalar_open ? launch_overlapped(k_update<true>, (int)nb, kThreads, 0, s, a)
+                                     : launch_overlapped(k_update<false>, (int)nb, kThreads, 0, s, a);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "launch of the update kernel");
+    ctx->scalar_open = false;
     ctx->launches += 1;
     ctx->last_stream = s;
     return ADASCALE_OK;
@@ -831,6 +878,8 @@ adascale_status adascale_apply_sums(adascale_ctx *ctx, const void *sums, const a
     cudaStream_t s = (cudaStream_t)cuda_stream;
     adascale_status st = sync_update_table(ctx, params, momentum, s);  // before anything is enqueued
     if (st != ADASCALE_OK) return st;
+    st = finish_open_scalar(ctx, s);
+    if (st != ADASCALE_OK) return st;
     ScalarArgs a;
     a.st = ctx->d_state;
     a.sums = static_cast<const double *>(sums);
@@ -875,6 +924,10 @@ adascale_status adascale_get_gain_tau(adascale_ctx *ctx, adascale_stats *out, in
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     CU(cudaStreamIsCapturing(s, &cap));
     if (cap != cudaStreamCaptureStatusNone) return ADASCALE_ERR_STATE;
+    {
+        adascale_status so = finish_open_scalar(ctx, s);  // a reduce launch with no update after it
+        if (so != ADASCALE_OK) return so;
+    }
     if (ctx->snap_inflight) {
         if (blocking) {
             CU(cudaEventSynchronize(ctx->ev_snap));
@@ -943,6 +996,10 @@ adascale_status adascale_get_state(adascale_ctx *ctx, void *buf)
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
     DevState d;
+    {
+        adascale_status so = finish_open_scalar(ctx, ctx->last_stream);
+        if (so != ADASCALE_OK) return so;
+    }
     CU(cudaStreamSynchronize(ctx->last_stream));
     CU(cudaMemcpy(&d, ctx->d_state, sizeof d, cudaMemcpyDeviceToHost));
     StateBlob b;
@@ -984,6 +1041,7 @@ adascale_status adascale_set_state(adascale_ctx *ctx, const void *buf)
     d.r = b.r;
     d.eta = b.eta;
     d.lr = b.lr;
+    ctx->scalar_open = false;  // the state is replaced as a whole: an iteration left open is dropped with it
     CU(cudaStreamSynchronize(ctx->last_stream));
     CU(cudaMemcpy(ctx->d_state, &d, sizeof d, cudaMemcpyHostToDevice));
     // a launch that gave up on a wait may have left its work counters half way

@@ -77,6 +77,12 @@ struct DevState {
 };
 static_assert(sizeof(DevState) == 112, "the snapshot copied to the host is 112 bytes");
 
+// What an iteration's scalar part reads of the state it starts from.
+struct RawState {
+    double tau, avg_a, avg_b;
+    long long n, t, skipped;
+};
+
 struct ScalarCfg {
     double eps, theta;  // theta already resolved on the host (the paper's rule follows S)
     unsigned flags;
@@ -129,6 +135,8 @@ struct ReduceArgs {
     u64 *tile_counter;        // runs handed out beyond each block's first; zero between launches
     DevState *st;
     double *sums_out;         // not null: write (D, N) there and leave the scalar part to k_scalar
+    RawState *snapshot;       // not null: the scalar part is left to the next kernel (see k_update): block 0
+                              // copies the state it will start from here, and no block stays behind
     unsigned spin_limit;      // bound of the producer / consumer handshake waits
     unsigned early_rows;      // non-zero: the gradient rows may be read before griddepcontrol.wait
     int S, T;
@@ -151,10 +159,26 @@ struct UpdateArgs {
     const TileDesc *tiles;    // tiles of kUpdateTile elements
     long long n_tiles;
     const float *gbar;
-    const DevState *st;
+    DevState *st;
     unsigned *next_tile;      // tiles handed out beyond each block's first; wraps to zero by itself
     int T;
     float rho, lambda;
+    // only when the reduce kernel left the scalar part of the iteration to this one
+    const double2 *partials;  // one pair per block of the reduce launch
+    int n_partials;
+    const RawState *snapshot; // the state the iteration starts from, copied by the reduce launch
+    ScalarCfg sc;
+    Sched sched;
+};
+
+// The scalar part as a kernel of one block, when no update follows a reduce launch that left it open.
+struct FinishArgs {
+    DevState *st;
+    const double2 *partials;
+    int n_partials;
+    const RawState *snapshot;
+    ScalarCfg sc;
+    Sched sched;
 };
 
 // Streaming 128-bit load (read once, evict first): used by the bandwidth probes.
@@ -249,98 +273,161 @@ __device__ double lr_eval(const Sched &s, double t)
 {
     if (s.kind == ADASCALE_LR_EXP) return s.eta0 * pow(s.decay, t / s.t_s1);
     if (s.kind == ADASCALE_LR_STEP) {
-        int passed = 0;
-        for (int i = 0; i < s.n; ++i) passed += (t > s.w[i]) ? 1 : 0;
-        return s.eta0 * pow(s.decay, (double)passed);
+        double f = 1.0;  // decay^(milestones passed), by repeated multiplication
+        for (int i = 0; i < s.n; ++i) f = (t > s.w[i]) ? f * s.decay : f;
+        return s.eta0 * f;
     }
     return s.eta0;
 }
 
-__device__ __forceinline__ double ema(double prev, double sample, double theta, long long n)
+// The scalar part of an iteration in two halves.  Everything that depends only on the state the
+// iteration starts from (the schedule's value at tau_t, the averaging weight, the gain of the lagged
+// form) can be worked out while the gradient rows are still being read; what is left once the two
+// sums are known is a handful of operations and one division.  Every path (the last block of the
+// reduce kernel, the update kernel, the scalar kernels) runs these same two functions.
+struct ScalarPrep {
+    RawState s;
+    double lr;       // lr(floor(tau_t)), App. B.1
+    double th;       // weight of the old average: min(theta, 1 - 1/n), plain mean of the first samples (App. B.3)
+    double r_prior;  // gain from the averages of prior iterations (r_0 = 1)
+    double inv_S, inv_Sm1;  // 1/S and 1/(S-1): the second half multiplies where the formulas divide
+};
+
+__device__ __forceinline__ RawState raw_state(const DevState *st)
 {
-    // plain mean of the first samples until the exponential weight takes over (App. B.3)
-    double warm = 1.0 - 1.0 / (double)n;
-    double th = theta < warm ? theta : warm;
-    return th * prev + (1.0 - th) * sample;
+    RawState s;
+    s.tau = st->tau;
+    s.avg_a = st->avg_a;
+    s.avg_b = st->avg_b;
+    s.n = st->n;
+    s.t = st->t;
+    s.skipped = st->skipped;
+    return s;
 }
 
-// Scalar part of the iteration: one thread, fp64, no host involvement.
-__device__ void scalar_step(DevState *st, const ScalarCfg &c, const Sched &sched, double D, double N)
+__device__ __forceinline__ bool same_state(const RawState &x, const RawState &y)
 {
-    st->D = D;
-    st->N = N;
-    if (__ldcg(&st->fault)) {  // a bounded wait gave up somewhere: the sums are incomplete, nothing is applied
-        st->skipped += 1;
-        st->eta = 0.0;
-        return;
+    return __double_as_longlong(x.tau) == __double_as_longlong(y.tau) &&
+           __double_as_longlong(x.avg_a) == __double_as_longlong(y.avg_a) &&
+           __double_as_longlong(x.avg_b) == __double_as_longlong(y.avg_b) && x.n == y.n && x.t == y.t &&
+           x.skipped == y.skipped;
+}
+
+__device__ ScalarPrep scalar_prepare(const RawState &s, const ScalarCfg &c, const Sched &sched)
+{
+    ScalarPrep p;
+    p.s = s;
+    const double t_arg = (c.flags & ADASCALE_FLAG_CONT_TAU) ? s.tau : floor(s.tau);
+    p.lr = lr_eval(sched, t_arg);
+    const double S = (double)c.S;
+    const double warm = 1.0 - 1.0 / (double)(s.n + 1);
+    p.th = c.theta < warm ? c.theta : warm;
+    p.inv_S = 1.0 / S;
+    p.inv_Sm1 = c.S > 1 ? 1.0 / (S - 1.0) : 0.0;
+    p.r_prior = 1.0;  // wanted by the lagged form only
+    if ((c.flags & ADASCALE_FLAG_LAGGED) && c.S > 1 && s.n > 0)
+        p.r_prior = (c.flags & ADASCALE_FLAG_RATIO) ? (s.avg_a + c.eps) / (s.avg_b + c.eps)
+                                                    : (s.avg_a + s.avg_b) / fma(s.avg_a, p.inv_S, s.avg_b);
+    return p;
+}
+
+// explicit roundings here and explicit fused operations below: the same value whichever kernel
+// the function is compiled into
+__device__ __forceinline__ double ema(double prev, double sample, double th)
+{
+    return __dadd_rn(__dmul_rn(th, prev), __dmul_rn(__dsub_rn(1.0, th), sample));
+}
+
+// Second half: from the two sums to r_t, eta_t, tau_{t+1}.  Returns eta_t (0 when the iteration is
+// skipped); writes the state when st is given.  One thread, fp64, no host involvement.
+__device__ double scalar_finish(DevState *st, const ScalarPrep &p, const ScalarCfg &c, double D, double N,
+                                             unsigned fault, bool &skip)
+{
+    if (st) {
+        st->D = D;
+        st->N = N;
+    }
+    skip = true;
+    if (fault) {  // a bounded wait gave up somewhere: the sums are incomplete, nothing is applied
+        if (st) {
+            st->skipped = p.s.skipped + 1;
+            st->eta = 0.0;
+        }
+        return 0.0;
     }
     if (!isfinite(D) || !isfinite(N)) {  // skip the iteration, leave every average and tau alone
-        st->status = ADASCALE_STATUS_NONFINITE;
-        st->skipped += 1;
-        st->eta = 0.0;
-        return;
+        if (st) {
+            st->status = ADASCALE_STATUS_NONFINITE;
+            st->skipped = p.s.skipped + 1;
+            st->eta = 0.0;
+        }
+        return 0.0;
     }
-    st->status = 0;
-    const double S = (double)c.S;
-    const double tau = st->tau;
-    const double t_arg = (c.flags & ADASCALE_FLAG_CONT_TAU) ? tau : floor(tau);
-    double r;
+    skip = false;
+    double r, sigma2_raw, mu2_raw, na = p.s.avg_a, nb = p.s.avg_b;
+    long long n = p.s.n;
     if (c.S == 1) {  // App. A.2: unit gain at scale one
-        st->sigma2_raw = 0.0;
-        st->mu2_raw = N;
+        sigma2_raw = 0.0;
+        mu2_raw = N;
         r = 1.0;
     } else {
-        double a, b, r_prior;
+        double a, b;
         const bool ratio = (c.flags & ADASCALE_FLAG_RATIO) != 0;
         if (ratio) {
             // Sec. 3.4: (1/S) sum_i ||g_i||^2 = D/S + N  and ||gbar||^2
-            a = D / S + N;
+            a = fma(D, p.inv_S, N);
             b = N;
-            st->sigma2_raw = a;
-            st->mu2_raw = b;
-            r_prior = st->n > 0 ? (st->avg_a + c.eps) / (st->avg_b + c.eps) : 1.0;
+            sigma2_raw = a;
+            mu2_raw = b;
         } else {
             // App. B.3: sigma^2 = D/(S-1) equals 1/(S-1) sum||g_i||^2 - S/(S-1)||gbar||^2
-            double sigma2 = D / (S - 1.0);
-            double mu2 = N - sigma2 / S;
-            st->sigma2_raw = sigma2;
-            st->mu2_raw = mu2;
+            const double sigma2 = D * p.inv_Sm1;
+            const double mu2 = fma(-sigma2, p.inv_S, N);
+            sigma2_raw = sigma2;
+            mu2_raw = mu2;
             a = sigma2 > c.eps ? sigma2 : c.eps;
             b = mu2 > 0.0 ? mu2 : 0.0;
-            r_prior = st->n > 0 ? (st->avg_a + st->avg_b) / (st->avg_a / S + st->avg_b) : 1.0;
         }
-        const long long n = st->n + 1;
-        const double na = ema(st->avg_a, a, c.theta, n);
-        const double nb = ema(st->avg_b, b, c.theta, n);
+        n = p.s.n + 1;
+        na = ema(p.s.avg_a, a, p.th);
+        nb = ema(p.s.avg_b, b, p.th);
+        if (c.flags & ADASCALE_FLAG_LAGGED)
+            r = p.r_prior;
+        else
+            r = ratio ? (na + c.eps) / (nb + c.eps) : (na + nb) / fma(na, p.inv_S, nb);  // Eq. 3
+    }
+    const double eta = r * p.lr;  // Sec. 3.2
+    if (st) {
+        st->status = 0;
+        st->sigma2_raw = sigma2_raw;
+        st->mu2_raw = mu2_raw;
         st->n = n;
         st->avg_a = na;
         st->avg_b = nb;
-        if (c.flags & ADASCALE_FLAG_LAGGED)
-            r = r_prior;
-        else
-            r = ratio ? (na + c.eps) / (nb + c.eps) : (na + nb) / (na / S + nb);  // Eq. 3
+        st->r = r;
+        st->lr = p.lr;
+        st->eta = eta;
+        st->tau = p.s.tau + r;
+        st->t = p.s.t + 1;
     }
-    const double lr = lr_eval(sched, t_arg);
-    st->r = r;
-    st->lr = lr;
-    st->eta = r * lr;     // Sec. 3.2
-    st->tau = tau + r;
-    st->t += 1;
+    return eta;
+}
+
+// Both halves in one go, on the state in place.
+__device__ void scalar_step(DevState *st, const ScalarCfg &c, const Sched &sched, double D, double N)
+{
+    const ScalarPrep p = scalar_prepare(raw_state(st), c, sched);
+    bool skip;
+    scalar_finish(st, p, c, D, N, __ldcg(&st->fault), skip);
 }
 
 // Lagged estimate (App. B.3: r_t from the averages of prior iterations only, r_0 = 1): the
-// learning rate of the coming iteration is known before its gradients are read.  Same
-// expressions as in scalar_step, so both give the identical value.
+// learning rate of the coming iteration is known before its gradients are read.  The same
+// first half as the scalar step's, so both give the identical value.
 __device__ double lagged_eta(const DevState *st, const ScalarCfg &c, const Sched &sched)
 {
-    const double S = (double)c.S;
-    double r = 1.0;
-    if (c.S > 1 && st->n > 0)
-        r = (c.flags & ADASCALE_FLAG_RATIO) ? (st->avg_a + c.eps) / (st->avg_b + c.eps)
-                                            : (st->avg_a + st->avg_b) / (st->avg_a / S + st->avg_b);
-    const double tau = st->tau;
-    const double t_arg = (c.flags & ADASCALE_FLAG_CONT_TAU) ? tau : floor(tau);
-    return r * lr_eval(sched, t_arg);
+    const ScalarPrep p = scalar_prepare(raw_state(st), c, sched);
+    return p.r_prior * p.lr;
 }
 
 // Programmatic dependent launch: a kernel lets its successor in the stream be scheduled
@@ -975,6 +1062,9 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
         // kernel allowed to start (see the ordering rule above).
         griddep_wait();
         trigger_early();
+        // the scalar part is left to the next kernel: it needs the state this iteration starts from,
+        // kept apart from the state that its block 0 will overwrite while other blocks still start
+        if (a.snapshot && blockIdx.x == 0 && tid == 0) *a.snapshot = raw_state(a.st);
         float eta = 0.f;
         if constexpr (FUSED) {
             if (tid == 0) eta_shared = (float)lagged_eta(a.st, a.sc, a.sched);
@@ -1183,6 +1273,12 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     if (tid == 0) {
         if (abort_flag) atomicOr(&a.st->fault, ADASCALE_STATUS_WAIT_TIMEOUT);
         a.partials[blockIdx.x] = make_double2(accD, accN);
+    }
+    // Scalar part left to the next kernel (small and mid-size jobs, static assignment): every block
+    // of that kernel adds up the pairs itself, so nothing here waits for the last block; the
+    // dependents are released when the last block exits, which is when every other SM is idle.
+    if (a.snapshot) return;
+    if (tid == 0) {
         __threadfence();
         const unsigned tk = atomicAdd(a.ticket, 1u);
         is_last = (tk == gridDim.x - 1);
@@ -1256,23 +1352,58 @@ __device__ __forceinline__ void update4(float4 &ww, float4 &vv, const float4 &gg
     ww.w = fmaf(-eta, vv.w, ww.w);
 }
 
-// A block's first tile is tile blockIdx.x; every further tile comes from a counter, so at any moment the blocks of the grid work on one
-// narrow, advancing window of the three arrays whatever the relative speed of the SMs (a
-// narrow window keeps DRAM pages and the read/write batches of the memory controller
-// efficient), and no SM idles at the end.  The counter value is fetched one tile ahead and the
+__device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
+// Adds the pairs p[0..n) in a fixed order with a block of kThreads threads; the sums are valid in thread 0.
+__device__ __forceinline__ void sum_pairs(const double2 *p, int n, double &d, double &nn, double *sa, double *sb)
+{
+    d = 0.0;
+    nn = 0.0;
+    for (int i = threadIdx.x; i < n; i += kThreads) {
+        const double2 e = __ldcg(&p[i]);
+        d += e.x;
+        nn += e.y;
+    }
+    block_sum2<kWarps>(d, nn, sa, sb);
+}
+
+// A block's first tile is tile blockIdx.x; every further tile comes from a counter, so at any
+// moment the blocks of the grid work on one narrow, advancing window of the three arrays
+// whatever the relative speed of the SMs (a narrow window keeps DRAM pages and the read/write
+// batches of the memory controller efficient), and no SM idles at the end.  The counter value is fetched one tile ahead and the
 // descriptor of the next tile while the current one is processed.  A tile is kUpdateTile =
 // 1024 * C elements: C 128-bit accesses per array and thread, all requested before the first
 // is used.  The counter needs no reset: every block asks once more than it gets tiles (its last
 // answer is the one that tells it to stop), so a launch asks exactly n_tiles times, and the
 // counter is an atomicInc that wraps to zero after n_tiles increments.
+//
+// DEFER: the reduce launch before this one stopped at one pair of sums per block, and every block
+// here completes the iteration's scalar part by itself: the same pairs, added in the same order,
+// give every block the same eta_t, and block 0 records the new state.  The first half of the
+// scalar part (schedule, averaging weight: most of its time) runs before the wait, on the state as
+// this block finds it; the state is only trusted if it equals, bit for bit, the copy that the
+// reduce launch made of it (a block that starts late may find the state already overwritten by
+// block 0, and then starts over from the copy).  The second half runs while the block's first
+// tile is on its way from memory into L2.  What the reduce kernel would spend after its last block has
+// finished - an exit ticket, one block adding up the pairs, one thread doing the scalar part,
+// about 5 us on the critical path of every iteration - is gone.
+template <bool DEFER>
 __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const __grid_constant__ UpdateArgs a)
 {
     constexpr int C = kUpdateVecs;
     __shared__ long long s_next[2];
+    __shared__ double sa[kWarps], sb[kWarps];
+    __shared__ float s_eta;
+    __shared__ int s_skip;
+    __shared__ ScalarPrep s_prep;
     const int tid = threadIdx.x, T = a.T;
     const long long n_tiles = a.n_tiles, G = gridDim.x;
     long long c = blockIdx.x;
     TileDesc d = {}, dn = {};
+    RawState found = {};
+    if constexpr (DEFER) {
+        if (tid == 0) found = raw_state(a.st);  // requested first, used after the tables below have arrived
+    }
     // Before the wait: only tables that the host wrote (descriptor, the tensor's pointers and flags).
     float *wq = nullptr, *vq = nullptr;
     unsigned fl = 0;
@@ -1282,18 +1413,62 @@ __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const _
         vq = (float *)a.wv[T + d.tensor];
         fl = a.wflags[d.tensor];
     }
+    if constexpr (DEFER) {
+        if (tid == 0) s_prep = scalar_prepare(found, a.sc, a.sched);  // thread 0's own use later
+    }
     griddep_wait();
     griddep_launch();
-    // a skipped iteration (non-finite sums, or a bounded wait that gave up) changes nothing; every
-    // block sees the same state, so either all of them ask the counter or none does
-    const bool skip = (a.st->status & ADASCALE_STATUS_NONFINITE) || a.st->fault;
-    if (skip) return;
-    const float eta = (float)a.st->eta;
+    float eta = 0.f;
+    if constexpr (!DEFER) {
+        // a skipped iteration (non-finite sums, or a bounded wait that gave up) changes nothing; every
+        // block sees the same state, so either all of them ask the counter or none does
+        const bool skip = (a.st->status & ADASCALE_STATUS_NONFINITE) || a.st->fault;
+        if (skip) return;
+        eta = (float)a.st->eta;
+    }
     // the counter belongs to the update launches; it is touched only after the wait, so that even
     // two update launches in a row cannot meet on it
     const unsigned wrap = (unsigned)(n_tiles - 1);
-    if (tid == 0) s_next[0] = G + (long long)atomicInc(a.next_tile, wrap);
-    __syncthreads();
+    unsigned asked = 0;  // thread 0: the counter's answer, looked at as late as possible
+    if (tid == 0) asked = atomicInc(a.next_tile, wrap);
+    if constexpr (DEFER) {
+        // The block's first tile is asked into L2 (no registers held), and the scalar part is
+        // completed while it travels.
+        RawState now = {};
+        unsigned fault = 0;
+        if (tid == 0) {  // requested before the pairs, used after them
+            now = *a.snapshot;
+            fault = __ldcg(&a.st->fault);
+        }
+        if (c < n_tiles) {
+            const int e = tid * 4 * C;  // this thread's first element of the tile
+            if (e < d.len) {
+                prefetch_l2(a.gbar + d.goff + e);
+                prefetch_l2(wq + d.first + e);
+                prefetch_l2(vq + d.first + e);
+            }
+        }
+        double D, N;
+        sum_pairs(a.partials, a.n_partials, D, N, sa, sb);
+        if (tid == 0) {
+            if (!same_state(now, s_prep.s)) s_prep = scalar_prepare(now, a.sc, a.sched);
+            bool skip;
+            s_eta = (float)scalar_finish(blockIdx.x == 0 ? a.st : nullptr, s_prep, a.sc, D, N, fault, skip);
+            s_skip = skip ? 1 : 0;
+            s_next[0] = G + (long long)asked;
+        }
+        __syncthreads();
+        eta = s_eta;
+        if (s_skip) {
+            // nothing is applied, but the counter must still see every request of this launch
+            if (tid == 0)
+                for (long long x = s_next[0]; x < n_tiles;) x = G + (long long)atomicInc(a.next_tile, wrap);
+            return;
+        }
+    } else {
+        if (tid == 0) s_next[0] = G + (long long)asked;
+        __syncthreads();
+    }
     int buf = 0;
     while (c < n_tiles) {
         const long long nc = s_next[buf];
@@ -1347,6 +1522,23 @@ __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const _
         c = nc;
         buf ^= 1;
         d = dn;
+    }
+}
+
+// The scalar part on its own, one block: when a reduce launch left it open and no update follows
+// (the caller asks for the statistics, or reduces again).  Same sums in the same order, same two
+// halves as in the update kernel, so the state is the same whichever of the two completes it.
+__global__ void __launch_bounds__(kThreads) k_finish(const __grid_constant__ FinishArgs a)
+{
+    __shared__ double sa[kWarps], sb[kWarps];
+    griddep_wait();
+    griddep_launch();
+    double D, N;
+    sum_pairs(a.partials, a.n_partials, D, N, sa, sb);
+    if (threadIdx.x == 0) {
+        const ScalarPrep prep = scalar_prepare(*a.snapshot, a.sc, a.sched);
+        bool skip;
+        scalar_finish(a.st, prep, a.sc, D, N, __ldcg(&a.st->fault), skip);
     }
 }
 

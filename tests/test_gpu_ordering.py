@@ -216,3 +216,102 @@ def test_set_state_clears_a_timeout():
     st = ada.get_gain_tau(True)
     assert st.status_bits == 0 and st.t == 2
     ada.close()
+
+
+# ---- the scalar part left open by a reduce launch -------------------------------------------
+
+def _small_job(seed, S=8, k=1.0):
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(seed)
+    numels = [30000, 4097, 64, 5]
+    m = [0.1 * torch.randn(n, device=DEV, generator=gen) for n in numels]
+    rows = [[m[j] + k * 0.1 * torch.randn(n, device=DEV, generator=gen) for j, n in enumerate(numels)] for _ in range(S)]
+    w = [torch.randn(n, device=DEV, generator=gen) for n in numels]
+    v = [torch.zeros(n, device=DEV) for n in numels]
+    return numels, rows, w, v
+
+
+def test_a_reduce_call_without_an_update_still_completes_its_iteration():
+    """On small jobs the reduce kernel stops at one pair of sums per block and the next kernel does
+    the scalar part: the update kernel when one follows, a one-block kernel when the caller asks
+    for the statistics (or reduces again) first.  Whichever completes it, the state is the same."""
+    numels, rows, w0, v0 = _small_job(77)
+    _, rows2, _, _ = _small_job(78, k=3.0)
+    sched = B.make_schedule("step", eta0=0.1, d=0.5, milestones=(1.0, 3.0))
+    kw = dict(momentum=0.9, weight_decay=1e-4)
+
+    ref = B.AdaScale(numels, 8, **kw)
+    w, v = [t.clone() for t in w0], [t.clone() for t in v0]
+    ref.step(rows, w, v, sched)
+    one = ref.get_gain_tau(True).as_dict()
+    w_one, v_one = [t.clone() for t in w], [t.clone() for t in v]
+    ref.step(rows2, w, v, sched)
+    two = ref.get_gain_tau(True).as_dict()
+    assert ref.launch_count == 4
+    ref.close()
+
+    # statistics asked for between the two halves: completed by the one-block kernel, then a plain update
+    ada = B.AdaScale(numels, 8, **kw)
+    w, v = [t.clone() for t in w0], [t.clone() for t in v0]
+    ada.reduce(rows, sched)
+    assert ada.get_gain_tau(True).as_dict() == one
+    assert ada.launch_count == 2
+    ada.update(w, v)
+    ada.update(w, v)        # a second update reads eta_t from the state and applies it once more
+    torch.cuda.synchronize()
+    assert ada.launch_count == 4
+    assert ada.get_gain_tau(True).as_dict() == one
+    ada.close()
+
+    ada = B.AdaScale(numels, 8, **kw)
+    w, v = [t.clone() for t in w0], [t.clone() for t in v0]
+    ada.reduce(rows, sched)
+    assert ada.get_gain_tau(True).t == 1
+    ada.update(w, v)
+    torch.cuda.synchronize()
+    for a, b in zip(w + v, w_one + v_one):
+        assert torch.equal(a, b)
+    ada.close()
+
+    # two reduce calls in a row: the first iteration is completed before the second starts
+    ada = B.AdaScale(numels, 8, **kw)
+    ada.reduce(rows, sched)
+    ada.reduce(rows2, sched)
+    assert ada.get_gain_tau(True).as_dict() == two
+    assert ada.launch_count == 4      # reduce, scalar, reduce, scalar
+    ada.close()
+
+    # a state set from outside replaces everything, an open iteration included
+    donor = B.AdaScale(numels, 8, **kw)
+    blob = donor.get_state()
+    donor.close()
+    ada = B.AdaScale(numels, 8, **kw)
+    ada.reduce(rows, sched)
+    ada.set_state(blob)
+    st = ada.get_gain_tau(True)
+    assert st.t == 0 and st.tau == 0.0
+    ada.reduce(rows, sched)
+    assert ada.get_gain_tau(True).as_dict()["r"] == one["r"]
+    ada.close()
+
+
+def test_the_open_scalar_part_and_the_last_block_form_agree():
+    """Runs from the counter keep the scalar part in the reduce kernel's last block; the static
+    assignment leaves it to the update kernel.  Same functions, sums in a different order."""
+    numels, rows, w0, v0 = _small_job(79, S=16)
+    sched = B.make_schedule("exp", eta0=0.1, d=0.5, T_S1=4.0)
+    out = []
+    for runs in (0, 2):
+        ada = B.AdaScale(numels, 16, momentum=0.9)
+        ada.set_tile_runs(runs)
+        w, v = [t.clone() for t in w0], [t.clone() for t in v0]
+        for _ in range(3):
+            ada.step(rows, w, v, sched)
+        out.append((ada.get_gain_tau(True), w, v))
+        ada.close()
+    a, b = out[0][0], out[1][0]
+    for f in ("r", "tau", "eta", "sigma2_raw", "mu2_raw", "sigma2_avg", "mu2_avg"):
+        assert abs(getattr(a, f) - getattr(b, f)) <= 1e-12 * abs(getattr(b, f)), f
+    assert a.t == b.t == 3
+    for x, y in zip(out[0][1] + out[0][2], out[1][1] + out[1][2]):
+        assert torch.allclose(x, y, rtol=1e-6, atol=1e-7)
