@@ -180,7 +180,6 @@ struct adascale_ctx {
     bool scalar_open = false;
     int open_pairs = 0;
     ScalarCfg open_sc;
-    Sched open_sched;
     PtrTable tg, tw;
     long long n_tiles = 0, n_stiles = 0;  // of the descriptors on the device
     DevState *h_snap = nullptr;  // pinned
@@ -507,9 +506,8 @@ adascale_status finish_open_scalar(adascale_ctx *ctx, cudaStream_t s)
     a.st = ctx->d_state;
     a.partials = ctx->d_partials;
     a.n_partials = ctx->open_pairs;
-    a.snapshot = reinterpret_cast<const RawState *>(ctx->d_ticket + 128);
+    a.prepared = reinterpret_cast<const ScalarPrep *>(ctx->d_ticket + 128);
     a.sc = ctx->open_sc;
-    a.sched = ctx->open_sched;
     cudaError_t e = launch_overlapped(k_finish, 1, kThreads, 0, s, a);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "launch of the scalar kernel");
     ctx->launches += 1;
@@ -558,7 +556,7 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
     // Static assignment, two-kernel form, sums not wanted by the caller: one pair per block is all
     // that is left to add up, and every block of the update kernel can do that itself.
     const bool leave_open = !fused && !sums_out && a.run_tiles == 0;
-    a.snapshot = leave_open ? reinterpret_cast<RawState *>(ctx->d_ticket + 128) : nullptr;
+    a.prepared = leave_open ? reinterpret_cast<ScalarPrep *>(ctx->d_ticket + 128) : nullptr;
     a.spin_limit = ctx->wait_spins;
     a.early_rows = (ctx->flags & ADASCALE_FLAG_GRADS_READY) ? 1u : 0u;
     a.S = S;
@@ -579,7 +577,6 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
         ctx->scalar_open = true;
         ctx->open_pairs = (int)nb;
         ctx->open_sc = a.sc;
-        ctx->open_sched = a.sched;
     }
     return ADASCALE_OK;
 }
@@ -632,9 +629,8 @@ adascale_status do_update(adascale_ctx *ctx, void *const *params, void *const *m
     a.lambda = (float)ctx->lambda;
     a.partials = ctx->d_partials;
     a.n_partials = ctx->open_pairs;
-    a.snapshot = reinterpret_cast<const RawState *>(ctx->d_ticket + 128);
+    a.prepared = reinterpret_cast<const ScalarPrep *>(ctx->d_ticket + 128);
     a.sc = ctx->open_sc;
-    a.sched = ctx->open_sched;
     long long nb = n_tiles;
     if (nb > (long long)ctx->sms * kUpdateBlocksPerSM) nb = (long long)ctx->sms * kUpdateBlocksPerSM;
     cudaError_t e = ctx->scalar_open ? launch_overlapped(k_update<true>, (int)nb, kThreads, 0, s, a)

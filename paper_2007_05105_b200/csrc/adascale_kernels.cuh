@@ -83,6 +83,15 @@ struct RawState {
     long long n, t, skipped;
 };
 
+// What the second half of the scalar part needs of the first (see scalar_prepare).
+struct ScalarPrep {
+    RawState s;
+    double lr;       // lr(floor(tau_t)), App. B.1
+    double th;       // weight of the old average: min(theta, 1 - 1/n), plain mean of the first samples (App. B.3)
+    double r_prior;  // gain from the averages of prior iterations (r_0 = 1)
+    double inv_S, inv_Sm1;  // 1/S and 1/(S-1): the second half multiplies where the formulas divide
+};
+
 struct ScalarCfg {
     double eps, theta;  // theta already resolved on the host (the paper's rule follows S)
     unsigned flags;
@@ -135,8 +144,8 @@ struct ReduceArgs {
     u64 *tile_counter;        // runs handed out beyond each block's first; zero between launches
     DevState *st;
     double *sums_out;         // not null: write (D, N) there and leave the scalar part to k_scalar
-    RawState *snapshot;       // not null: the scalar part is left to the next kernel (see k_update): block 0
-                              // copies the state it will start from here, and no block stays behind
+    ScalarPrep *prepared;     // not null: the scalar part is left to the next kernel (see k_update): block 0
+                              // leaves its first half here, and no block stays behind at the end
     unsigned spin_limit;      // bound of the producer / consumer handshake waits
     unsigned early_rows;      // non-zero: the gradient rows may be read before griddepcontrol.wait
     int S, T;
@@ -166,9 +175,8 @@ struct UpdateArgs {
     // only when the reduce kernel left the scalar part of the iteration to this one
     const double2 *partials;  // one pair per block of the reduce launch
     int n_partials;
-    const RawState *snapshot; // the state the iteration starts from, copied by the reduce launch
+    const ScalarPrep *prepared;  // first half of the scalar part, left by the reduce launch
     ScalarCfg sc;
-    Sched sched;
 };
 
 // The scalar part as a kernel of one block, when no update follows a reduce launch that left it open.
@@ -176,9 +184,8 @@ struct FinishArgs {
     DevState *st;
     const double2 *partials;
     int n_partials;
-    const RawState *snapshot;
+    const ScalarPrep *prepared;
     ScalarCfg sc;
-    Sched sched;
 };
 
 // Streaming 128-bit load (read once, evict first): used by the bandwidth probes.
@@ -285,13 +292,6 @@ __device__ double lr_eval(const Sched &s, double t)
 // form) can be worked out while the gradient rows are still being read; what is left once the two
 // sums are known is a handful of operations and one division.  Every path (the last block of the
 // reduce kernel, the update kernel, the scalar kernels) runs these same two functions.
-struct ScalarPrep {
-    RawState s;
-    double lr;       // lr(floor(tau_t)), App. B.1
-    double th;       // weight of the old average: min(theta, 1 - 1/n), plain mean of the first samples (App. B.3)
-    double r_prior;  // gain from the averages of prior iterations (r_0 = 1)
-    double inv_S, inv_Sm1;  // 1/S and 1/(S-1): the second half multiplies where the formulas divide
-};
 
 __device__ __forceinline__ RawState raw_state(const DevState *st)
 {
@@ -305,12 +305,16 @@ __device__ __forceinline__ RawState raw_state(const DevState *st)
     return s;
 }
 
-__device__ __forceinline__ bool same_state(const RawState &x, const RawState &y)
+// What another kernel left for this one, read from L2.
+__device__ __forceinline__ ScalarPrep load_prepared(const ScalarPrep *q)
 {
-    return __double_as_longlong(x.tau) == __double_as_longlong(y.tau) &&
-           __double_as_longlong(x.avg_a) == __double_as_longlong(y.avg_a) &&
-           __double_as_longlong(x.avg_b) == __double_as_longlong(y.avg_b) && x.n == y.n && x.t == y.t &&
-           x.skipped == y.skipped;
+    static_assert(sizeof(ScalarPrep) == 11 * 8, "eleven 8-byte fields");
+    ScalarPrep p;
+    const long long *src = reinterpret_cast<const long long *>(q);
+    long long *dst = reinterpret_cast<long long *>(&p);
+#pragma unroll
+    for (int i = 0; i < 11; ++i) dst[i] = __ldcg(src + i);
+    return p;
 }
 
 __device__ ScalarPrep scalar_prepare(const RawState &s, const ScalarCfg &c, const Sched &sched)
@@ -1062,9 +1066,11 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
         // kernel allowed to start (see the ordering rule above).
         griddep_wait();
         trigger_early();
-        // the scalar part is left to the next kernel: it needs the state this iteration starts from,
-        // kept apart from the state that its block 0 will overwrite while other blocks still start
-        if (a.snapshot && blockIdx.x == 0 && tid == 0) *a.snapshot = raw_state(a.st);
+        // The scalar part is left to the next kernel.  Its first half needs only the state this
+        // iteration starts from: one thread works it out here, while the block's first rows are
+        // still on their way, and leaves it where every block of the next kernel will read it
+        // (apart from the state itself, which that kernel's block 0 overwrites while others start).
+        if (a.prepared && blockIdx.x == 0 && tid == 0) *a.prepared = scalar_prepare(raw_state(a.st), a.sc, a.sched);
         float eta = 0.f;
         if constexpr (FUSED) {
             if (tid == 0) eta_shared = (float)lagged_eta(a.st, a.sc, a.sched);
@@ -1277,7 +1283,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     // Scalar part left to the next kernel (small and mid-size jobs, static assignment): every block
     // of that kernel adds up the pairs itself, so nothing here waits for the last block; the
     // dependents are released when the last block exits, which is when every other SM is idle.
-    if (a.snapshot) return;
+    if (a.prepared) return;
     if (tid == 0) {
         __threadfence();
         const unsigned tk = atomicAdd(a.ticket, 1u);
@@ -1380,11 +1386,10 @@ __device__ __forceinline__ void sum_pairs(const double2 *p, int n, double &d, do
 // DEFER: the reduce launch before this one stopped at one pair of sums per block, and every block
 // here completes the iteration's scalar part by itself: the same pairs, added in the same order,
 // give every block the same eta_t, and block 0 records the new state.  The first half of the
-// scalar part (schedule, averaging weight: most of its time) runs before the wait, on the state as
-// this block finds it; the state is only trusted if it equals, bit for bit, the copy that the
-// reduce launch made of it (a block that starts late may find the state already overwritten by
-// block 0, and then starts over from the copy).  The second half runs while the block's first
-// tile is on its way from memory into L2.  What the reduce kernel would spend after its last block has
+// scalar part (schedule, averaging weight: most of its time) was done by the reduce launch while
+// it waited for its first rows, and is read from where it left it (not from the state, which
+// block 0 may already have overwritten when a block starts late).  The second half runs while
+// the block's first tile is on its way from memory into L2.  What the reduce kernel would spend after its last block has
 // finished - an exit ticket, one block adding up the pairs, one thread doing the scalar part,
 // about 5 us on the critical path of every iteration - is gone.
 template <bool DEFER>
@@ -1400,10 +1405,6 @@ __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const _
     const long long n_tiles = a.n_tiles, G = gridDim.x;
     long long c = blockIdx.x;
     TileDesc d = {}, dn = {};
-    RawState found = {};
-    if constexpr (DEFER) {
-        if (tid == 0) found = raw_state(a.st);  // requested first, used after the tables below have arrived
-    }
     // Before the wait: only tables that the host wrote (descriptor, the tensor's pointers and flags).
     float *wq = nullptr, *vq = nullptr;
     unsigned fl = 0;
@@ -1412,9 +1413,6 @@ __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const _
         wq = (float *)a.wv[d.tensor];
         vq = (float *)a.wv[T + d.tensor];
         fl = a.wflags[d.tensor];
-    }
-    if constexpr (DEFER) {
-        if (tid == 0) s_prep = scalar_prepare(found, a.sc, a.sched);  // thread 0's own use later
     }
     griddep_wait();
     griddep_launch();
@@ -1434,10 +1432,9 @@ __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const _
     if constexpr (DEFER) {
         // The block's first tile is asked into L2 (no registers held), and the scalar part is
         // completed while it travels.
-        RawState now = {};
         unsigned fault = 0;
         if (tid == 0) {  // requested before the pairs, used after them
-            now = *a.snapshot;
+            s_prep = load_prepared(a.prepared);
             fault = __ldcg(&a.st->fault);
         }
         if (c < n_tiles) {
@@ -1451,7 +1448,6 @@ __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const _
         double D, N;
         sum_pairs(a.partials, a.n_partials, D, N, sa, sb);
         if (tid == 0) {
-            if (!same_state(now, s_prep.s)) s_prep = scalar_prepare(now, a.sc, a.sched);
             bool skip;
             s_eta = (float)scalar_finish(blockIdx.x == 0 ? a.st : nullptr, s_prep, a.sc, D, N, fault, skip);
             s_skip = skip ? 1 : 0;
@@ -1536,7 +1532,7 @@ __global__ void __launch_bounds__(kThreads) k_finish(const __grid_constant__ Fin
     double D, N;
     sum_pairs(a.partials, a.n_partials, D, N, sa, sb);
     if (threadIdx.x == 0) {
-        const ScalarPrep prep = scalar_prepare(*a.snapshot, a.sc, a.sched);
+        const ScalarPrep prep = load_prepared(a.prepared);
         bool skip;
         scalar_finish(a.st, prep, a.sc, D, N, __ldcg(&a.st->fault), skip);
     }

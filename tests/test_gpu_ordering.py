@@ -220,7 +220,7 @@ def test_set_state_clears_a_timeout():
 
 # ---- the scalar part left open by a reduce launch -------------------------------------------
 
-def _small_job(seed, S=8, k=1.0):
+def _open_job(seed, S=8, k=1.0):
     gen = torch.Generator(device=DEV)
     gen.manual_seed(seed)
     numels = [30000, 4097, 64, 5]
@@ -235,8 +235,8 @@ def test_a_reduce_call_without_an_update_still_completes_its_iteration():
     """On small jobs the reduce kernel stops at one pair of sums per block and the next kernel does
     the scalar part: the update kernel when one follows, a one-block kernel when the caller asks
     for the statistics (or reduces again) first.  Whichever completes it, the state is the same."""
-    numels, rows, w0, v0 = _small_job(77)
-    _, rows2, _, _ = _small_job(78, k=3.0)
+    numels, rows, w0, v0 = _open_job(77)
+    _, rows2, _, _ = _open_job(78, k=3.0)
     sched = B.make_schedule("step", eta0=0.1, d=0.5, milestones=(1.0, 3.0))
     kw = dict(momentum=0.9, weight_decay=1e-4)
 
@@ -298,7 +298,7 @@ def test_a_reduce_call_without_an_update_still_completes_its_iteration():
 def test_the_open_scalar_part_and_the_last_block_form_agree():
     """Runs from the counter keep the scalar part in the reduce kernel's last block; the static
     assignment leaves it to the update kernel.  Same functions, sums in a different order."""
-    numels, rows, w0, v0 = _small_job(79, S=16)
+    numels, rows, w0, v0 = _open_job(79, S=16)
     sched = B.make_schedule("exp", eta0=0.1, d=0.5, T_S1=4.0)
     out = []
     for runs in (0, 2):
