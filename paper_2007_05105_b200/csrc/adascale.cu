@@ -556,7 +556,8 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
     // Static assignment, two-kernel form, sums not wanted by the caller: one pair per block is all
     // that is left to add up, and every block of the update kernel can do that itself.
     const bool leave_open = !fused && !sums_out && a.run_tiles == 0;
-    a.prepared = leave_open ? reinterpret_cast<ScalarPrep *>(ctx->d_ticket + 128) : nullptr;
+    a.prepared = reinterpret_cast<ScalarPrep *>(ctx->d_ticket + 128);
+    a.leave_open = leave_open ? 1u : 0u;
     a.spin_limit = ctx->wait_spins;
     a.early_rows = (ctx->flags & ADASCALE_FLAG_GRADS_READY) ? 1u : 0u;
     a.S = S;

@@ -144,8 +144,8 @@ struct ReduceArgs {
     u64 *tile_counter;        // runs handed out beyond each block's first; zero between launches
     DevState *st;
     double *sums_out;         // not null: write (D, N) there and leave the scalar part to k_scalar
-    ScalarPrep *prepared;     // not null: the scalar part is left to the next kernel (see k_update): block 0
-                              // leaves its first half here, and no block stays behind at the end
+    ScalarPrep *prepared;     // block 0 leaves the first half of the scalar part here, for whoever runs the second
+    unsigned leave_open;      // non-zero: that is the next kernel (see k_update), and no block stays behind at the end
     unsigned spin_limit;      // bound of the producer / consumer handshake waits
     unsigned early_rows;      // non-zero: the gradient rows may be read before griddepcontrol.wait
     int S, T;
@@ -423,15 +423,6 @@ __device__ void scalar_step(DevState *st, const ScalarCfg &c, const Sched &sched
     const ScalarPrep p = scalar_prepare(raw_state(st), c, sched);
     bool skip;
     scalar_finish(st, p, c, D, N, __ldcg(&st->fault), skip);
-}
-
-// Lagged estimate (App. B.3: r_t from the averages of prior iterations only, r_0 = 1): the
-// learning rate of the coming iteration is known before its gradients are read.  The same
-// first half as the scalar step's, so both give the identical value.
-__device__ double lagged_eta(const DevState *st, const ScalarCfg &c, const Sched &sched)
-{
-    const ScalarPrep p = scalar_prepare(raw_state(st), c, sched);
-    return p.r_prior * p.lr;
 }
 
 // Programmatic dependent launch: a kernel lets its successor in the stream be scheduled
@@ -713,6 +704,11 @@ __device__ __forceinline__ u64 l2_keep_policy()
     return p;
 }
 
+__device__ __forceinline__ void store_pair_keep(double2 *p, double x, double y, u64 policy)
+{
+    asm volatile("st.global.L2::cache_hint.v2.f64 [%0], {%1, %2}, %3;" ::"l"(p), "d"(x), "d"(y), "l"(policy) : "memory");
+}
+
 template <int CPT>
 __device__ __forceinline__ void store_cols_keep(float *g, const float *m, u64 policy)
 {
@@ -829,6 +825,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     if (producer) {
         u64 policy;
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+        const u64 keep_pairs = l2_keep_policy();  // the run pairs are read once more, by the last block
         int last_use[kStages];
 #pragma unroll
         for (int i = 0; i < kStages; ++i) last_use[i] = -1;
@@ -919,7 +916,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                 const long long tile = slot == 0 ? qt0 : (slot == 1 ? qt1 : (slot == 2 ? qt2 : qt3));
                 if ((tile + 1) % R == 0 || tile + 1 == n_tiles) {  // last tile of its run
                     const double D = warp_sum(runD), N = warp_sum(runN);
-                    if (lane == 0) a.run_partials[tile / R] = make_double2(D, N);
+                    if (lane == 0) store_pair_keep(&a.run_partials[tile / R], D, N, keep_pairs);
                     runD = runN = 0.0;
                 }
             }
@@ -1066,16 +1063,23 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
         // kernel allowed to start (see the ordering rule above).
         griddep_wait();
         trigger_early();
-        // The scalar part is left to the next kernel.  Its first half needs only the state this
-        // iteration starts from: one thread works it out here, while the block's first rows are
-        // still on their way, and leaves it where every block of the next kernel will read it
-        // (apart from the state itself, which that kernel's block 0 overwrites while others start).
-        if (a.prepared && blockIdx.x == 0 && tid == 0) *a.prepared = scalar_prepare(raw_state(a.st), a.sc, a.sched);
+        // The first half of the scalar part needs only the state this iteration starts from: one
+        // thread of block 0 works it out here, while the block's first rows are still on their way,
+        // and leaves it for whoever runs the second half: the last block of this launch, or every
+        // block of the next kernel (which must not read the state itself: its block 0 overwrites
+        // the state while other blocks may still be starting).
         float eta = 0.f;
         if constexpr (FUSED) {
-            if (tid == 0) eta_shared = (float)lagged_eta(a.st, a.sc, a.sched);
+            // one-pass form: eta_t of the lagged estimate is the product of two of its values
+            if (tid == 0) {
+                const ScalarPrep prep = scalar_prepare(raw_state(a.st), a.sc, a.sched);
+                eta_shared = (float)(prep.r_prior * prep.lr);
+                if (blockIdx.x == 0) *a.prepared = prep;
+            }
             asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");  // consumers only
             eta = eta_shared;
+        } else {
+            if (blockIdx.x == 0 && tid == 0) *a.prepared = scalar_prepare(raw_state(a.st), a.sc, a.sched);
         }
         constexpr int NP = CPT / 2;
         const u64 keep = l2_keep_policy();
@@ -1283,7 +1287,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     // Scalar part left to the next kernel (small and mid-size jobs, static assignment): every block
     // of that kernel adds up the pairs itself, so nothing here waits for the last block; the
     // dependents are released when the last block exits, which is when every other SM is idle.
-    if (a.prepared) return;
+    if (a.leave_open) return;
     if (tid == 0) {
         __threadfence();
         const unsigned tk = atomicAdd(a.ticket, 1u);
@@ -1295,6 +1299,9 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
 
     // Last stage, fixed order: thread j adds the pairs j, j+288, ... of the runs in index order,
     // sixteen loads in flight at a time, then the per-block pairs likewise, then the block tree.
+    // (The run pairs were stored with the evict-last priority, so they are still in L2.  Bringing
+    // them in through the idle stages with bulk copies was measured too: 14 against 11 us for
+    // 30 K pairs, one SM cannot keep more bytes in flight that way than with these loads.)
     __threadfence();
     double d = 0.0, n = 0.0;
     const long long n_pairs = a.run_tiles > 0 ? (n_tiles + a.run_tiles - 1) / a.run_tiles : 0;
@@ -1325,7 +1332,8 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
             a.sums_out[0] = d;
             a.sums_out[1] = n;
         } else {
-            scalar_step(a.st, a.sc, a.sched, d, n);
+            bool skip;
+            scalar_finish(a.st, load_prepared(a.prepared), a.sc, d, n, __ldcg(&a.st->fault), skip);
         }
         *a.ticket = 0u;
         *a.tile_counter = 0ull;
