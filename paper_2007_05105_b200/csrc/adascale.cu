@@ -553,9 +553,10 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
     a.tile_counter = reinterpret_cast<u64 *>(ctx->d_ticket + 192);
     a.st = ctx->d_state;
     a.sums_out = sums_out;
-    // Static assignment, two-kernel form, sums not wanted by the caller: one pair per block is all
-    // that is left to add up, and every block of the update kernel can do that itself.
-    const bool leave_open = !fused && !sums_out && a.run_tiles == 0;
+    // Two-kernel form, sums not wanted by the caller: the reduce kernel stops at its pairs of sums.
+    // Static assignment: one pair per block, which every block of the update kernel adds up itself.
+    // Runs from the counter: a small kernel first brings the run pairs down to a few dozen.
+    const bool leave_open = !fused && !sums_out;
     a.prepared = reinterpret_cast<ScalarPrep *>(ctx->d_ticket + 128);
     a.leave_open = leave_open ? 1u : 0u;
     a.spin_limit = ctx->wait_spins;
@@ -578,6 +579,20 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
         ctx->scalar_open = true;
         ctx->open_pairs = (int)nb;
         ctx->open_sc = a.sc;
+        if (a.run_tiles > 0) {
+            SumArgs sa;
+            sa.run_partials = ctx->d_run_partials;
+            sa.n_pairs = (n_tiles + a.run_tiles - 1) / a.run_tiles;
+            sa.out = ctx->d_partials + nb;
+            sa.tile_counter = a.tile_counter;
+            long long sb = (sa.n_pairs + kThreads - 1) / kThreads;
+            if (sb > kSumBlocks) sb = kSumBlocks;
+            if (sb < 1) sb = 1;
+            e = launch_overlapped(k_sum, (int)sb, kThreads, 0, s, sa);
+            if (e != cudaSuccess) return cuda_fail(ctx, e, "launch of the pair-sum kernel");
+            ctx->launches += 1;
+            ctx->open_pairs = (int)(nb + sb);
+        }
     }
     return ADASCALE_OK;
 }
@@ -777,7 +792,7 @@ adascale_status adascale_init(const adascale_config *cfg, adascale_ctx **out)
         const size_t gbar_alloc = (g > 0 && !(ctx->flags & ADASCALE_FLAG_FUSED)) ? (size_t)g : 1;
         CU(cudaMalloc(&ctx->d_gbar, gbar_alloc * sizeof(float)));
         CU(cudaMemset(ctx->d_gbar, 0, gbar_alloc * sizeof(float)));
-        CU(cudaMalloc(&ctx->d_partials, (size_t)(ctx->sms * kReduceBlocksPerSM + 1) * sizeof(double2)));
+        CU(cudaMalloc(&ctx->d_partials, (size_t)(ctx->sms * kReduceBlocksPerSM + kSumBlocks + 1) * sizeof(double2)));
         CU(cudaMalloc(&ctx->d_run_partials,
                       (size_t)(rcap + ctx->sms * kReduceBlocksPerSM + 1) * sizeof(double2)));
         CU(cudaMalloc(&ctx->d_ticket, 4 * 256));  // counters, 256 bytes apart: exit ticket, update tiles, (spare), runs

@@ -49,6 +49,7 @@ constexpr int kUpdateBlocksPerSM = 4;
 constexpr long long kDynamicMinTiles = 32768;  // staged tiles from which they are handed out from a counter
 constexpr int kSlots = kStages + 1;       // tiles of a block whose sums can be on their way at once
 static_assert(kSlots == 4, "the producer keeps the tile index of each slot in four named registers");
+constexpr int kSumBlocks = 64;            // blocks of the kernel that adds up the run pairs of a large job
 constexpr int kScalarTile = 2048;         // elements per tile on the unaligned / ragged-tail path
 constexpr int kUpdateTile = 1024 * kUpdateVecs;  // elements per tile of the update kernel
 constexpr int kGbarAlign = 64;            // every tensor's mean gradient starts on a 256-byte boundary
@@ -177,6 +178,14 @@ struct UpdateArgs {
     int n_partials;
     const ScalarPrep *prepared;  // first half of the scalar part, left by the reduce launch
     ScalarCfg sc;
+};
+
+// First level of the sum over the run pairs of a large job (see k_sum).
+struct SumArgs {
+    const double2 *run_partials;
+    long long n_pairs;
+    double2 *out;        // one pair per block of the launch
+    u64 *tile_counter;   // the reduce launch's run counter, put back to zero here
 };
 
 // The scalar part as a kernel of one block, when no update follows a reduce launch that left it open.
@@ -1321,12 +1330,20 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
             n += p.y;
         }
     }
-    for (int i = tid; i < (int)gridDim.x; i += kStagedThreads) {
-        const double2 p = __ldcg(&a.partials[i]);
-        d += p.x;
-        n += p.y;
+    block_sum2<kStagedWarps>(d, n, sa, sb);  // the run pairs (zero with the static assignment)
+    // The per-block pairs in the order in which sum_pairs adds them (the producer warp adds zeros), so
+    // that this form and the one that leaves the scalar part to the update kernel agree bit for bit.
+    double db = 0.0, nb = 0.0;
+    if (tid < kThreads) {
+        for (int i = tid; i < (int)gridDim.x; i += kThreads) {
+            const double2 p = __ldcg(&a.partials[i]);
+            db += p.x;
+            nb += p.y;
+        }
     }
-    block_sum2<kStagedWarps>(d, n, sa, sb);
+    block_sum2<kStagedWarps>(db, nb, sa, sb);
+    d = db + d;
+    n = nb + n;
     if (tid == 0) {
         if (a.sums_out) {  // sharded use: the caller adds the shards' sums, k_scalar continues
             a.sums_out[0] = d;
@@ -1526,6 +1543,32 @@ __global__ void __launch_bounds__(kThreads, kUpdateBlocksPerSM) k_update(const _
         c = nc;
         buf ^= 1;
         d = dn;
+    }
+}
+
+// Large jobs leave tens of thousands of run pairs.  One block (the reduce kernel's last) needs
+// 10-17 us to add them up, with every other SM idle; a few dozen blocks need one round of loads.
+// Block b adds the pairs of slice b, thread j the pairs j, j + 256, ... of the slice, then the
+// block tree: a fixed order, whatever ran where.  The pairs of this launch join the per-block
+// pairs of the reduce launch, and the update kernel (or k_finish) adds up both.
+__global__ void __launch_bounds__(kThreads) k_sum(const __grid_constant__ SumArgs a)
+{
+    __shared__ double sa[kWarps], sb[kWarps];
+    griddep_wait();
+    griddep_launch();
+    const long long per = (a.n_pairs + gridDim.x - 1) / gridDim.x;
+    const long long first = (long long)blockIdx.x * per;
+    const long long end = first + per < a.n_pairs ? first + per : a.n_pairs;
+    double d = 0.0, n = 0.0;
+    for (long long i = first + threadIdx.x; i < end; i += kThreads) {
+        const double2 e = __ldcg(&a.run_partials[i]);
+        d += e.x;
+        n += e.y;
+    }
+    block_sum2<kWarps>(d, n, sa, sb);
+    if (threadIdx.x == 0) {
+        a.out[blockIdx.x] = make_double2(d, n);
+        if (blockIdx.x == 0) *a.tile_counter = 0ull;
     }
 }
 

@@ -315,3 +315,30 @@ def test_the_open_scalar_part_and_the_last_block_form_agree():
     assert a.t == b.t == 3
     for x, y in zip(out[0][1] + out[0][2], out[1][1] + out[1][2]):
         assert torch.allclose(x, y, rtol=1e-6, atol=1e-7)
+
+
+def test_large_job_form_with_the_pair_sum_kernel():
+    """Runs from the counter in the two-kernel form: reduce, a small kernel that adds up the run pairs, update
+    (three launches per step); a reduce call that no update follows is completed by the one-block kernel."""
+    numels, rows, w0, v0 = _open_job(81, S=16)
+    sched = B.make_schedule("const", eta0=0.05)
+    ref = B.AdaScale(numels, 16, momentum=0.9)
+    ref.set_tile_runs(2)
+    w, v = [t.clone() for t in w0], [t.clone() for t in v0]
+    ref.step(rows, w, v, sched)
+    torch.cuda.synchronize()
+    assert ref.launch_count == 3
+    one = ref.get_gain_tau(True).as_dict()
+    ref.close()
+
+    ada = B.AdaScale(numels, 16, momentum=0.9)
+    ada.set_tile_runs(2)
+    w2, v2 = [t.clone() for t in w0], [t.clone() for t in v0]
+    ada.reduce(rows, sched)
+    assert ada.get_gain_tau(True).as_dict() == one
+    assert ada.launch_count == 3       # reduce, pair sum, scalar
+    ada.update(w2, v2)
+    torch.cuda.synchronize()
+    for a, b in zip(w + v, w2 + v2):
+        assert torch.equal(a, b)
+    ada.close()
