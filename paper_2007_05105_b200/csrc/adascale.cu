@@ -549,14 +549,28 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
     // Two stages in flight per block are enough and measured 2-5 % faster than three when tiles are
     // assigned statically; with runs from a counter three were 2 % faster.
     a.stages = a.run_tiles > 0 ? (unsigned)kStages : 2u;
+    // Runs of run_tiles tiles, except at the end of the launch: the tiles of the last runs (two per
+    // block, but no more than half of all) are handed out one by one, so that the blocks finish
+    // within a tile of each other.
+    a.long_runs = 0;
+    if (a.run_tiles > 0) {
+        const long long n_full = n_tiles / a.run_tiles;
+        long long singles = 2LL * max_blocks;
+        if (singles > n_full / 2) singles = n_full / 2;
+        a.long_runs = n_full - singles;
+    }
+    const long long n_run_pairs = a.run_tiles > 0 ? a.long_runs + (n_tiles - a.long_runs * a.run_tiles) : 0;
     a.ticket = ctx->d_ticket;
     a.tile_counter = reinterpret_cast<u64 *>(ctx->d_ticket + 192);
     a.st = ctx->d_state;
     a.sums_out = sums_out;
-    // Two-kernel form, sums not wanted by the caller: the reduce kernel stops at its pairs of sums.
-    // Static assignment: one pair per block, which every block of the update kernel adds up itself.
-    // Runs from the counter: a small kernel first brings the run pairs down to a few dozen.
-    const bool leave_open = !fused && !sums_out;
+    // Sums not wanted by the caller: the reduce kernel stops at its pairs of sums.  Two-kernel form,
+    // static assignment: one pair per block, which every block of the update kernel adds up itself.
+    // Runs from the counter: a small kernel first brings the run pairs down to a few dozen; in the
+    // one-pass form, where no update kernel follows, the one-block scalar kernel comes right after
+    // it (with the static assignment the one-pass form keeps its last block: the next launch's
+    // blocks are then already waiting on the SMs when the scalar part ends).
+    const bool leave_open = !sums_out && (!fused || a.run_tiles > 0);
     a.prepared = reinterpret_cast<ScalarPrep *>(ctx->d_ticket + 128);
     a.leave_open = leave_open ? 1u : 0u;
     a.spin_limit = ctx->wait_spins;
@@ -582,7 +596,7 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
         if (a.run_tiles > 0) {
             SumArgs sa;
             sa.run_partials = ctx->d_run_partials;
-            sa.n_pairs = (n_tiles + a.run_tiles - 1) / a.run_tiles;
+            sa.n_pairs = n_run_pairs;
             sa.out = ctx->d_partials + nb;
             sa.tile_counter = a.tile_counter;
             long long sb = (sa.n_pairs + kThreads - 1) / kThreads;
@@ -593,6 +607,7 @@ adascale_status do_reduce(adascale_ctx *ctx, const void *const *grads, const ada
             ctx->launches += 1;
             ctx->open_pairs = (int)(nb + sb);
         }
+        if (fused) return finish_open_scalar(ctx, s);
     }
     return ADASCALE_OK;
 }

@@ -140,6 +140,7 @@ struct ReduceArgs {
     double2 *partials;        // [grid] sums over each block's scalar-path tiles
     double2 *run_partials;    // sums of the staged tiles, one pair per run (run_tiles > 0)
     long long run_tiles;      // consecutive staged tiles handed out together; 0: static assignment
+    long long long_runs;      // the first long_runs runs have run_tiles tiles, every later run a single tile
     unsigned stages;          // shared-memory stages in use, 2 .. kStages
     unsigned *ticket;
     u64 *tile_counter;        // runs handed out beyond each block's first; zero between launches
@@ -852,7 +853,13 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
         // miss delays a copy.
         const long long G = gridDim.x;
         const long long R = a.run_tiles;       // 0: static assignment
-        const long long n_runs = R > 0 ? (n_tiles + R - 1) / R : 0;
+        // The last runs of a launch are single tiles: what the blocks differ by when the counter runs
+        // dry is then one tile, not one run (10-20 us of idle SMs at the end of a large job).
+        const long long A = a.long_runs, AR = A * R;
+        const long long n_runs = R > 0 ? A + (n_tiles - AR) : 0;
+        auto run_first = [&](long long r) -> long long { return r < A ? r * R : AR + (r - A); };
+        auto run_of = [&](long long tile) -> long long { return tile < AR ? tile / R : A + (tile - AR); };
+        auto run_ends = [&](long long tile) -> bool { return tile >= AR || (tile + 1) % R == 0; };
         // Before its wait this warp only reads tables that the host wrote (descriptors, row pointers:
         // their uploads are full stream dependencies), so the first tile's addresses are ready when
         // the wait returns.  The rows are the caller's data: unless the caller has vouched that
@@ -874,7 +881,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
         auto next_tile = [&](long long tile) -> long long {
             if (tile >= n_tiles) return n_tiles;
             if (R == 0) return tile + G < n_tiles ? tile + G : n_tiles;
-            if ((tile + 1) % R != 0 && tile + 1 < n_tiles) return tile + 1;
+            if (!run_ends(tile)) return tile + 1;
             const long long r = rq0;
             rq0 = rq1;
             if (late_fetch || r >= n_runs) {
@@ -883,13 +890,13 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
                 rq1 = take_asked();
                 if (rq1 < n_runs) ask_run();
             }
-            return r < n_runs ? r * R : n_tiles;
+            return r < n_runs ? run_first(r) : n_tiles;
         };
         TileDesc d0, d1 = {}, d2 = {};
         const char *rowptr = nullptr, *rowptr_n = nullptr;
         float *pw = nullptr, *pv = nullptr, *pw_n = nullptr, *pv_n = nullptr;  // fused mode, lane 0 only
         unsigned pfl = 0, pfl_n = 0;
-        long long t = R > 0 ? ((long long)blockIdx.x < n_runs ? (long long)blockIdx.x * R : n_tiles)
+        long long t = R > 0 ? ((long long)blockIdx.x < n_runs ? run_first(blockIdx.x) : n_tiles)
                             : ((long long)blockIdx.x < n_tiles ? (long long)blockIdx.x : n_tiles);
         long long t1 = next_tile(t);
         if (t < n_tiles) d1 = a.tiles[t];
@@ -923,9 +930,9 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
             }
             if (R > 0) {
                 const long long tile = slot == 0 ? qt0 : (slot == 1 ? qt1 : (slot == 2 ? qt2 : qt3));
-                if ((tile + 1) % R == 0 || tile + 1 == n_tiles) {  // last tile of its run
+                if (run_ends(tile)) {
                     const double D = warp_sum(runD), N = warp_sum(runN);
-                    if (lane == 0) store_pair_keep(&a.run_partials[tile / R], D, N, keep_pairs);
+                    if (lane == 0) store_pair_keep(&a.run_partials[run_of(tile)], D, N, keep_pairs);
                     runD = runN = 0.0;
                 }
             }
@@ -1313,7 +1320,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     // 30 K pairs, one SM cannot keep more bytes in flight that way than with these loads.)
     __threadfence();
     double d = 0.0, n = 0.0;
-    const long long n_pairs = a.run_tiles > 0 ? (n_tiles + a.run_tiles - 1) / a.run_tiles : 0;
+    const long long n_pairs = a.run_tiles > 0 ? a.long_runs + (n_tiles - a.long_runs * a.run_tiles) : 0;
     {
         constexpr int U = 16;
         long long i = tid;
