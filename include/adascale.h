@@ -149,7 +149,9 @@ adascale_status adascale_init(const adascale_config *cfg, adascale_ctx **out);
 
 /*
  * One iteration (Sec. 3.2, App. B.3, Eq. 2-3): reduce + update, two kernel launches on
- * `cuda_stream` (a cudaStream_t passed as void*, NULL = default stream).  Returns after
+ * `cuda_stream` (a cudaStream_t passed as void*, NULL = default stream); three for jobs whose
+ * tiles are handed out in runs (see adascale_tiling), where a small kernel between the two
+ * adds up the partial sums of the runs.  Returns after
  * enqueueing.  It waits for the device in one case only: when the tiling has to be rebuilt
  * (first call, a new S, a tensor whose 16-byte alignment changed) the tile descriptors are
  * uploaded and the call waits for that upload.
@@ -175,10 +177,10 @@ adascale_status adascale_step(adascale_ctx *ctx, const void *const *grads, void 
  * First half of adascale_step: streams the S x P gradient matrix once, writes gbar,
  * forms sum_i ||g_i - gbar||^2 and ||gbar||^2 and runs the scalar part (estimates,
  * averages, r_t, eta_t, tau_{t+1}) on the device (Sec. 3.2, App. B.3, Eq. 3).
- * Arguments as in adascale_step.  One kernel launch.
- * Where the scalar part runs is the library's business: for jobs whose tiles are assigned
- * statically (see adascale_tiling) the reduce kernel stops at one pair of sums per block
- * and the kernel that follows completes the iteration - the update kernel of
+ * Arguments as in adascale_step.  One kernel launch, two when the tiles are handed out in runs.
+ * Where the scalar part runs is the library's business: the reduce kernel stops at pairs of
+ * partial sums (one per block; with runs, one per run, brought down to a few dozen by a small
+ * second kernel) and the kernel that follows completes the iteration - the update kernel of
  * adascale_update / adascale_step, each of whose blocks adds up the pairs itself, or, when
  * adascale_get_gain_tau, adascale_get_state, adascale_apply_sums or another adascale_reduce
  * comes first, a one-block kernel that the library enqueues before serving that call (one
@@ -251,7 +253,8 @@ adascale_status adascale_set_wait_limit(adascale_ctx *ctx, uint32_t polls);
  * How the reduce kernel hands its tiles to the blocks, for the following steps: run_tiles = -1
  * (default) lets the library choose by the job's size (see adascale_tiling); 0 assigns tile t to
  * block t mod grid; 1 .. 64 hands out runs of that many consecutive tiles from a device
- * counter.  Every setting gives sums that are reproducible from run to run; different settings
+ * counter (the tiles of the last runs of a launch - two runs per block, at most half of all -
+ * one by one).  Every setting gives sums that are reproducible from run to run; different settings
  * add the same terms in different orders and so may differ in the last bits.  It exists for
  * tests (so that small jobs can exercise the path of large ones) and for tuning.  No counterpart
  * in the paper.  Errors: INVALID_ARG.
@@ -294,10 +297,10 @@ adascale_status adascale_stream_probe(int32_t kind, void *a, void *b, int64_t n_
  * staged tiles before each tensor into tprefix[0..n_tensors] and of scalar-path tiles into
  * sprefix[0..n_tensors], the columns of one staged tile into *tile_cols and the rows of one
  * shared-memory stage into *rows.  With fewer than 32768 staged tiles, or S <= 8, tile t is
- * processed by block t mod gridDim; larger jobs hand runs of 2 or 4 consecutive tiles to the
- * blocks as they become free, and the sums are added up per run and then over the runs in
- * index order, so the result does not depend on which block processed which run (see
- * adascale_set_tile_runs).  Makes no CUDA call.  Errors: INVALID_ARG.
+ * processed by block t mod gridDim; larger jobs hand runs of 2 or 4 consecutive tiles (single
+ * tiles at the end of a launch) to the blocks as they become free, and the sums are added up
+ * per run and then over the runs in a fixed order, so the result does not depend on which block
+ * processed which run (see adascale_set_tile_runs).  Makes no CUDA call.  Errors: INVALID_ARG.
  */
 adascale_status adascale_tiling(const int64_t *numel, int32_t n_tensors, int32_t grad_dtype, int32_t S,
                                 const uint8_t *aligned, int32_t n_blocks, int64_t *tprefix, int64_t *sprefix,
