@@ -40,7 +40,7 @@ HEADLINE = "decoder_24l"
 # captures summarised under profiles/ (None where no capture of the current kernel exists).
 # decoder_24l is too large to capture; its figure is the capture of a narrower decoder of the
 # same structure scaled by the number of parameters.
-NCU_TRAFFIC_BYTES = {"decoder_24l": 4.575e9 * 354823168 / 68212736, "decoder_4l": 4.575e9, "resnet50": 848.1e6}
+NCU_TRAFFIC_BYTES = {"decoder_24l": 4.578e9 * 354823168 / 68212736, "decoder_4l": 4.578e9, "resnet50": 850.8e6}
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 L2_BYTES = 126 * 1024 * 1024
