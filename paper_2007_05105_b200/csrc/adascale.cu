@@ -489,7 +489,7 @@ adascale_status sync_reduce_table(adascale_ctx *ctx, const void *const *grads, c
 
 // Staged tiles handed out together by the reduce kernel; 0 = static assignment (tile t to block
 // t mod grid).  Handing tiles out from a counter pays on large jobs only (it keeps all blocks on
-// one narrow window of the matrix); runs keep the number of pairs that the last block adds up small.
+// one narrow window of the matrix); runs keep the number of pairs to add up afterwards small.
 long long run_tiles_for(long long n_tiles, int S)
 {
     // tiles of a single row chunk (S <= 8) are too short for the producer warp's extra work per tile:
@@ -810,7 +810,8 @@ adascale_status adascale_init(const adascale_config *cfg, adascale_ctx **out)
         CU(cudaMalloc(&ctx->d_partials, (size_t)(ctx->sms * kReduceBlocksPerSM + kSumBlocks + 1) * sizeof(double2)));
         CU(cudaMalloc(&ctx->d_run_partials,
                       (size_t)(rcap + ctx->sms * kReduceBlocksPerSM + 1) * sizeof(double2)));
-        CU(cudaMalloc(&ctx->d_ticket, 4 * 256));  // counters, 256 bytes apart: exit ticket, update tiles, (spare), runs
+        // counters and scratch, 256 bytes apart: exit ticket, update tiles, prepared scalar part, runs
+        CU(cudaMalloc(&ctx->d_ticket, 4 * 256));
         CU(cudaMemset(ctx->d_ticket, 0, 4 * 256));
         CU(cudaMalloc(&ctx->d_state, sizeof(DevState)));
         CU(cudaMemset(ctx->d_state, 0, sizeof(DevState)));

@@ -5,10 +5,15 @@
 //   reduce  - streams the S x P gradient matrix once through shared memory (bulk asynchronous
 //             copies completed on mbarriers, a producer warp and eight consumer warps), writes
 //             the mean gradient and pairs (sum of squared deviations, squared norm of the mean)
-//             per block or per run of tiles; the block that finishes last adds the pairs in
-//             index order and runs the scalar part (estimates, clamps, moving averages, r_t,
-//             eta_t, tau_{t+1}).
-//   update  - v <- rho v + (gbar + lambda w), w <- w - eta_t v, reading eta_t from the device.
+//             per block or per run of tiles, and prepares the part of the scalar step that
+//             depends only on the state the iteration starts from.
+//   update  - every block adds up the pairs (for large jobs a 64-block kernel, k_sum, has brought
+//             them down to a few dozen first) and completes the scalar part (estimates, clamps,
+//             moving averages, r_t, eta_t, tau_{t+1}); then v <- rho v + (gbar + lambda w),
+//             w <- w - eta_t v.
+// Where no update kernel follows (one-pass form, sharded form, a reduce call on its own) the
+// pairs are added up and the scalar part completed by the reduce kernel's last block or by the
+// one-block kernels k_finish / k_scalar.
 // Three trivial streaming kernels calibrate the bandwidth ceiling.
 // The path is bound by HBM bandwidth; there is no contraction, hence no tensor-core work.
 //
@@ -810,8 +815,9 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     // returned.  Two-kernel mode: the successor is the update kernel, and a block of it that lands
     // on an SM where a reduce block still runs keeps that SM's split of shared memory and L1
     // (hardly any L1) for its whole life, which costs the update kernel up to a quarter of its
-    // speed; so only the block that finishes last triggers it, when every other SM is already
-    // idle, and the launch still overlaps the last stage below.
+    // speed; so the dependents are released only when every other SM is already idle: by the
+    // exit of the last block, or, where a last block stays behind to add up the pairs, by that
+    // block before it does so.
     auto trigger_early = [] {
         if constexpr (FUSED) griddep_launch();
     };
@@ -835,7 +841,7 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
     if (producer) {
         u64 policy;
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-        const u64 keep_pairs = l2_keep_policy();  // the run pairs are read once more, by the last block
+        const u64 keep_pairs = l2_keep_policy();  // the run pairs are read once more, right after this kernel
         int last_use[kStages];
 #pragma unroll
         for (int i = 0; i < kStages; ++i) last_use[i] = -1;
@@ -913,9 +919,9 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
         // in.  The consumers leave the 256 per-thread pairs of a tile in shared memory; lane l of
         // this warp adds threads l, l+32, ... of every tile of a run, in order, into its own fp64
         // pair; a shuffle tree adds the lanes at the end of the run and the result goes to
-        // run_partials[run] with a plain store.  The block that finishes last adds those pairs in
-        // index order, so nothing depends on which block processed which run.  (Static assignment:
-        // none of this; the consumer threads keep their own fp64 pairs, see below.)
+        // run_partials[run] with a plain store.  Whoever adds those pairs up (k_sum, or the block that
+        // finishes last) does so in a fixed order, so nothing depends on which block processed which
+        // run.  (Static assignment: none of this; the consumer threads keep their own fp64 pairs.)
         unsigned q = 0;                 // tiles this block has staged
         long long qt0 = 0, qt1 = 0, qt2 = 0, qt3 = 0;  // their indices, by slot (kSlots = 4)
         double runD = 0.0, runN = 0.0;  // this lane's share of the run being delivered
@@ -1057,8 +1063,9 @@ __global__ void __launch_bounds__(kStagedThreads, kReduceBlocksPerSM) k_reduce(c
         for (unsigned seq = q >= (unsigned)kSlots ? q - kSlots + 1 : 0u; R > 0 && seq < q && !timed_out; ++seq)
             if (!deliver(seq)) timed_out = true;
         // The answer to the last question put to the counter must have arrived before this block
-        // takes its exit ticket: the block that finishes last resets the counter, and an increment
-        // still on its way would land after the reset.  (Looking at the value makes the warp wait.)
+        // leaves: the counter is reset once all blocks have (by k_sum, or by the block that takes the
+        // last exit ticket), and an increment still on its way would land after the reset.  (Looking
+        // at the value makes the warp wait.)
         if (R > 0 && take_asked() < 0) timed_out = true;
         if (timed_out) atomicExch(&abort_flag, 1);
         // Every copy this warp has issued must have landed before the block may leave (its shared
