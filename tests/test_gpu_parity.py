@@ -604,10 +604,12 @@ def test_fused_mode_with_elastic_scale_host_gradients_and_resume():
     pair.close()
 
 
-def test_two_column_shards_reproduce_the_unsharded_step():
+@pytest.mark.parametrize("runs", [-1, 2])
+def test_two_column_shards_reproduce_the_unsharded_step(runs):
     """Column-sharded use emulated on one GPU: two contexts over the two halves of the tensor
     list, their sums added on the device (what an all-reduce of 16 bytes would do), then the
-    scalar part and the update per shard.  No kernel waits for another: the calls are sequential."""
+    scalar part and the update per shard.  No kernel waits for another: the calls are sequential.
+    With runs forced, the shards' reduce kernels keep a last block that adds up the run pairs."""
     gen = _gen(4400)
     numels = [30000, 4097, 64, 7, 2048, 12345]
     split = 3
@@ -622,6 +624,8 @@ def test_two_column_shards_reproduce_the_unsharded_step():
     ws, vs = _params(numels, _gen(4401))
     shards = [B.AdaScale(numels[:split], 8, momentum=0.9, weight_decay=1e-3),
               B.AdaScale(numels[split:], 8, momentum=0.9, weight_decay=1e-3)]
+    for ada in shards:
+        ada.set_tile_runs(runs)
     parts = [slice(0, split), slice(split, len(numels))]
     sums = [torch.zeros(2, dtype=torch.float64, device=DEV) for _ in shards]
     for i, rows in enumerate(steps):
